@@ -1,0 +1,166 @@
+/*
+ * libtrl — HRD policy-gradient scoring path for sm_100a (B200), C ABI.
+ *
+ * The calls follow the statement of the objective in Section 2.3 of the TritonRL paper
+ * ("Policy Optimization with Hierarchical Reward Decomposition"):
+ *
+ *   J(theta)   = E_i [ alpha J^plan_i + J^code_i ]
+ *   J^c_i      = (1/G) sum_j (1/|o_ij|) sum_{t in T^c_ij} min[ A^c_ij s_ijt , A^c_ij clip(s_ijt, 1-eps, 1+eps) ]
+ *   s_ijt      = pi_theta(o_ijt | .) / pi_theta_old(o_ijt | .)
+ *   A^c_ij     = r^c_ij - (1/G) sum_j r^c_ij ,   r^plan = R^speedup, r^code = R^correct   (Eq. 2)
+ *
+ * Shapes.  P prompts, G rollouts per prompt, B = P*G rollouts, each right-padded to T
+ * response tokens; N = B*T rows, row n = b*T + t.  len[b] in [0,T] is |o_ij|, bnd[b] in
+ * [0,len[b]] is the index of the first code token (t < bnd: plan segment; bnd <= t < len:
+ * code segment).  hidden[n,:] (H values) is the final hidden state that predicts token
+ * ids[n]; W is the LM head, [V,H] row-major, no bias, temperature 1.
+ *
+ * Conventions.
+ *  - Every pointer is a DEVICE pointer owned by the caller unless a comment says "host".
+ *    The library allocates no device memory and keeps no state between calls; scratch
+ *    comes from a caller-provided workspace of at least trl_workspace_bytes(...) bytes,
+ *    256-byte aligned.  Workspaces may be reused between calls on the same stream.
+ *  - All work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = default
+ *    stream).  Calls return without synchronising.
+ *  - Return value: TRL_OK or an error found on the host (bad argument, shape, workspace,
+ *    CUDA launch error).  Errors found on the device (token id outside [0,V), len outside
+ *    [0,T], bnd outside [0,len], a pipeline wait that ran out) are OR-ed as bit
+ *    (1 << code) into *status_dev (int32, caller zero-initialises it; may be NULL).  Offending rows
+ *    are treated as padding / clamped, so no out-of-bounds access happens.
+ *  - Outputs for padded rows (t >= len[b]) are defined: 0.
+ *  - Row-major everywhere.  bf16 tensors need H % 8 == 0 and V % 8 == 0 (16-byte rows).
+ */
+#ifndef TRL_H_
+#define TRL_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  TRL_OK = 0,
+  TRL_ERR_INVALID_ARG = 1,
+  TRL_ERR_SHAPE = 2,
+  TRL_ERR_DTYPE = 3,
+  TRL_ERR_WORKSPACE_TOO_SMALL = 4,
+  TRL_ERR_ARCH = 5,       /* device is not compute capability 10.x */
+  TRL_ERR_CUDA = 6,       /* a CUDA runtime / driver call failed   */
+  TRL_ERR_BAD_INDEX = 7,  /* device-detected: id, len or bnd out of range */
+  TRL_ERR_TIMEOUT = 8     /* device-detected: a bounded pipeline wait expired */
+} trl_status;
+
+/* Storage type of hidden / W / dHidden.  TRL_BF16 runs on the tcgen05 tensor cores with
+ * fp32 accumulation; TRL_F32 runs fp32 CUDA-core kernels (small problems, second opinion). */
+typedef enum { TRL_F32 = 0, TRL_BF16 = 1 } trl_dtype;
+
+typedef enum {
+  TRL_CALL_TOKEN_LOGPROBS = 0,
+  TRL_CALL_PG_LOSS_FWD = 1,
+  TRL_CALL_PG_LOSS_BWD = 2
+} trl_call;
+
+/* Hyper-parameters of the surrogate.  The paper uses eps_lo = eps_hi = 0.2 (training
+ * details appendix) and alpha = 0.1 (Section 3.1); alpha weights the plan term. */
+typedef struct {
+  float eps_lo;   /* lower clip: ratio clipped at 1 - eps_lo */
+  float eps_hi;   /* upper clip: ratio clipped at 1 + eps_hi */
+  float alpha;    /* weight of J^plan; J^code has weight 1   */
+} trl_pg_config;
+
+/* Bytes of workspace the given call wants for these shapes (recommended size).
+ * trl_pg_loss_bwd accepts any workspace >= trl_workspace_bytes_min(...) and processes rows
+ * in as many chunks as the workspace allows; larger is faster up to the recommended size.
+ * Returns 0 for an unknown call or invalid shape. */
+size_t trl_workspace_bytes(int which_call, int B, int T, int H, int V, trl_dtype dt);
+size_t trl_workspace_bytes_min(int which_call, int B, int T, int H, int V, trl_dtype dt);
+
+/*
+ * Token scoring: log pi(o_t | .) of the sampled tokens under one model (Section 2.3, the
+ * token probabilities in the ratio s_ijt).  Call once with the current policy's
+ * (hidden, W) and once with the old policy's ("reference model" in the uniform-reward
+ * appendix) to obtain logp and old_logp.
+ *
+ *   z[n,v] = sum_k hidden[n,k] W[v,k];  lse[n] = log sum_v exp z[n,v];  logp[n] = z[n,ids[n]] - lse[n]
+ *
+ * The [N,V] logits are never written to memory (bf16 path: vocabulary tiles are reduced
+ * to a running (max, sum-exp) pair in the GEMM epilogue).
+ *
+ * in : hidden [B*T,H] dt; W [V,H] dt; ids [B*T] int32; len [B] int32
+ * out: logp [B*T] f32; lse [B*T] f32 (save lse for trl_pg_loss_bwd)
+ */
+int trl_token_logprobs(const void* hidden, const void* W, const int32_t* ids, const int32_t* len,
+                       int B, int T, int H, int V, trl_dtype dt,
+                       float* logp, float* lse,
+                       void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream);
+
+/*
+ * Hierarchical Reward Decomposition (Section 2.3, Eq. 2 and the sentence before it):
+ * per-class group-relative advantages, segment labels and per-token advantages.
+ *
+ *   A_plan[b] = r_plan[b] - mean over the G rollouts of the same prompt (same for A_code)
+ *   seg[n] = 1 (plan) if t < bnd[b]; 2 (code) if bnd[b] <= t < len[b]; 0 (padding)
+ *   adv[n] = A_plan[b] / A_code[b] / 0 accordingly
+ *   n_plan[b] = bnd[b]; n_code[b] = len[b] - bnd[b]; *n_valid = sum_b len[b]
+ *
+ * adv_mode 0: A = r - mean (the paper).  adv_mode 1: A = (r - mean) / (population std + 1e-6)
+ * (not in the paper; the common GRPO normalisation).  Group means are taken in fp64, so a
+ * group of identical rewards gives exactly 0.
+ *
+ * in : r_plan, r_code [P*G] f32; len, bnd [P*G] int32
+ * out: A_plan, A_code [P*G] f32; seg [P*G*T] u8; adv [P*G*T] f32; n_plan, n_code [P*G] int32;
+ *      n_valid [1] int64.  Needs no workspace.
+ */
+int trl_hrd_advantages(const float* r_plan, const float* r_code,
+                       const int32_t* len, const int32_t* bnd, int P, int G, int T, int adv_mode,
+                       float* A_plan, float* A_code, uint8_t* seg, float* adv,
+                       int32_t* n_plan, int32_t* n_code, int64_t* n_valid,
+                       int32_t* status_dev, void* stream);
+
+/*
+ * Clipped surrogate (Section 2.3, the two displayed equations for J and J^c):
+ *
+ *   s = exp(logp - old_logp);  u = min(adv*s, adv*clip(s, 1-eps_lo, 1+eps_hi))
+ *   loss = -(1/P) sum_i (1/G) sum_j (1/len_ij) sum_{t<len_ij} w_t u_t,  w = alpha (plan), 1 (code)
+ *   g[n] = d loss / d logp[n] = -w adv s / (P G len) where the unclipped branch is the min, else 0
+ *
+ * Both classes are divided by the whole response length |o_ij| = len.  The sum is taken in
+ * a fixed order (bit-reproducible).
+ *
+ * in : logp, old_logp, adv [P*G*T] f32; seg [P*G*T] u8; len [P*G] int32
+ * out: loss [1] f32; g [P*G*T] f32 (0 on padding);
+ *      stats [4] f32 or NULL: fraction of valid tokens with s > 1+eps_hi, fraction with
+ *      s < 1-eps_lo, mean s, number of valid tokens.
+ */
+int trl_pg_loss_fwd(const float* logp, const float* old_logp, const float* adv, const uint8_t* seg,
+                    const int32_t* len, int P, int G, int T, trl_pg_config cfg,
+                    float* loss, float* g, float* stats,
+                    void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream);
+
+/*
+ * Backward of the loss to the LM-head inputs (the paper differentiates the objective of
+ * Section 2.3 automatically; this is the chain rule through logp = z[ids] - lse):
+ *
+ *   dS[n,v] = g[n] (1[v = ids[n]] - exp(z[n,v] - lse[n]))      (softmax recomputed from lse)
+ *   dHidden = dS W        dW = dS^T hidden
+ *
+ * dS exists only for one chunk of rows at a time inside the workspace.
+ *
+ * in : hidden, W, ids, len as in trl_token_logprobs; lse [B*T] f32 from it; g [B*T] f32
+ * out: dHidden [B*T,H] dt (padded rows 0); dW [V,H] f32 (overwritten)
+ */
+int trl_pg_loss_bwd(const void* hidden, const void* W, const int32_t* ids, const int32_t* len,
+                    const float* lse, const float* g,
+                    int B, int T, int H, int V, trl_dtype dt,
+                    void* dHidden, float* dW,
+                    void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream);
+
+/* Host string for a status code (static storage). */
+const char* trl_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TRL_H_ */

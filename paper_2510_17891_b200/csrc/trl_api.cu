@@ -1,0 +1,275 @@
+// extern "C" entry points of libtrl: argument checks, workspace carving, kernel sequencing.
+#include <cstring>
+
+#include "trl_internal.h"
+
+using namespace trl;
+
+namespace {
+
+constexpr int kRecommendedChunkRowsBf16 = 32768;
+constexpr int kRecommendedChunkRowsF32 = 2048;
+constexpr int kRasterBandFwd = 32;
+constexpr int kRasterBandBwd = 16;
+
+int check_device() {
+  static int cached = -1;
+  if (cached >= 0) return cached;
+  int dev = 0, major = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return TRL_ERR_CUDA;
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return TRL_ERR_CUDA;
+  cached = (major == 10) ? TRL_OK : TRL_ERR_ARCH;
+  return cached;
+}
+
+bool shapes_ok(int B, int T, int H, int V) {
+  return B > 0 && T > 0 && H > 0 && V > 0 && (long)B * T < (1L << 31) && (long)V * H < (1L << 40);
+}
+
+struct Carver {
+  char* base; size_t off = 0;
+  explicit Carver(void* p) : base((char*)p) {}
+  template <class Tp> Tp* take(size_t n) {
+    Tp* r = (Tp*)(base + off);
+    off += align_up(n * sizeof(Tp), 256);
+    return r;
+  }
+};
+
+size_t fwd_bytes_bf16(int B, int T, int V) {
+  const size_t rows_cap = (size_t)B * cdiv(T, kRowBlock) * kRowBlock;
+  const size_t nt = cdiv(V, 256);
+  return row_blocks_bytes(B, T) + align_up(rows_cap * 4, 256) + align_up(nt * rows_cap * 8, 256);
+}
+size_t fwd_bytes_f32(int B, int T, int H, int V, int R) {
+  return row_blocks_bytes(B, T) + align_up((size_t)R * H * 4, 256) + align_up((size_t)R * V * 4, 256);
+}
+size_t bwd_fixed_bf16(int B, int T, int H, int V) { return row_blocks_bytes(B, T) + align_up((size_t)H * V * 2, 256); }
+size_t bwd_per_rows_bf16(int H, int V, int R) {
+  return align_up((size_t)H * R * 2, 256) + 2 * align_up((size_t)R * V * 2, 256);
+}
+size_t bwd_bytes_f32(int B, int T, int H, int V, int R) {
+  return row_blocks_bytes(B, T) + 2 * align_up((size_t)R * H * 4, 256) + align_up((size_t)R * V * 4, 256);
+}
+int rows_cap_of(int B, int T) { return B * cdiv(T, kRowBlock) * kRowBlock; }
+
+// largest multiple of 128 rows (<= cap) whose scratch fits into `avail` bytes
+template <class F>
+int fit_rows(size_t avail, int cap, F bytes_of) {
+  int lo = 0, hi = cap / kRowBlock;
+  while (lo < hi) {
+    int mid = (lo + hi + 1) / 2;
+    if (bytes_of(mid * kRowBlock) <= avail) lo = mid; else hi = mid - 1;
+  }
+  return lo * kRowBlock;
+}
+
+size_t ws_bytes(int which, int B, int T, int H, int V, trl_dtype dt, bool minimum) {
+  if (!shapes_ok(B, T, H, V)) return 0;
+  if (dt != TRL_F32 && dt != TRL_BF16) return 0;
+  const int cap = rows_cap_of(B, T);
+  switch (which) {
+    case TRL_CALL_TOKEN_LOGPROBS:
+      if (dt == TRL_BF16) return fwd_bytes_bf16(B, T, V);
+      return fwd_bytes_f32(B, T, H, V, minimum ? kRowBlock : (cap < kRecommendedChunkRowsF32 ? cap : kRecommendedChunkRowsF32));
+    case TRL_CALL_PG_LOSS_FWD:
+      return align_up((size_t)B * pg_loss_tiles(T) * 4 * sizeof(float), 256);
+    case TRL_CALL_PG_LOSS_BWD:
+      if (dt == TRL_BF16) {
+        const int R = minimum ? kRowBlock : (cap < kRecommendedChunkRowsBf16 ? cap : kRecommendedChunkRowsBf16);
+        return bwd_fixed_bf16(B, T, H, V) + bwd_per_rows_bf16(H, V, R);
+      }
+      return bwd_bytes_f32(B, T, H, V, minimum ? kRowBlock : (cap < kRecommendedChunkRowsF32 ? cap : kRecommendedChunkRowsF32));
+  }
+  return 0;
+}
+
+#define TRL_CUDA_OK(expr) do { if ((expr) != cudaSuccess) return TRL_ERR_CUDA; } while (0)
+
+}  // namespace
+
+extern "C" {
+
+size_t trl_workspace_bytes(int which_call, int B, int T, int H, int V, trl_dtype dt) {
+  return ws_bytes(which_call, B, T, H, V, dt, false);
+}
+size_t trl_workspace_bytes_min(int which_call, int B, int T, int H, int V, trl_dtype dt) {
+  return ws_bytes(which_call, B, T, H, V, dt, true);
+}
+
+const char* trl_status_string(int status) {
+  switch (status) {
+    case TRL_OK: return "ok";
+    case TRL_ERR_INVALID_ARG: return "invalid argument";
+    case TRL_ERR_SHAPE: return "invalid shape";
+    case TRL_ERR_DTYPE: return "unsupported dtype";
+    case TRL_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case TRL_ERR_ARCH: return "device is not sm_100";
+    case TRL_ERR_CUDA: return "CUDA error";
+    case TRL_ERR_BAD_INDEX: return "index out of range (device)";
+    case TRL_ERR_TIMEOUT: return "pipeline wait timed out (device)";
+  }
+  return "unknown status";
+}
+
+int trl_token_logprobs(const void* hidden, const void* W, const int32_t* ids, const int32_t* len,
+                       int B, int T, int H, int V, trl_dtype dt, float* logp, float* lse,
+                       void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream) {
+  if (!hidden || !W || !ids || !len || !logp || !lse || !workspace) return TRL_ERR_INVALID_ARG;
+  if (dt != TRL_F32 && dt != TRL_BF16) return TRL_ERR_DTYPE;
+  if (!shapes_ok(B, T, H, V)) return TRL_ERR_SHAPE;
+  if (dt == TRL_BF16 && ((H % 8) || (V % 8))) return TRL_ERR_SHAPE;
+  if (((uintptr_t)workspace & 255) != 0) return TRL_ERR_INVALID_ARG;
+  if (workspace_bytes < trl_workspace_bytes_min(TRL_CALL_TOKEN_LOGPROBS, B, T, H, V, dt)) return TRL_ERR_WORKSPACE_TOO_SMALL;
+  if (int e = check_device()) return e;
+  cudaStream_t s = (cudaStream_t)stream;
+  const int cap_rows = rows_cap_of(B, T);
+
+  Carver cv(workspace);
+  RowBlocks rb = carve_row_blocks(cv.take<char>(row_blocks_bytes(B, T)), B, T);
+  launch_build_row_blocks(len, B, T, rb, status_dev, s);
+
+  if (dt == TRL_BF16) {
+    const int nt = cdiv(V, 256);
+    float* tgt = cv.take<float>(cap_rows);
+    float2* partials = cv.take<float2>((size_t)nt * cap_rows);
+    TcGemm g;
+    memset(&g, 0, sizeof(g));
+    g.epi = TC_EPI_LSE;
+    g.A = hidden; g.a_rows = (long)B * T; g.a_ld = H;
+    g.B = W; g.b_rows = V; g.b_ld = H;
+    g.K = H; g.N = V;
+    g.rb = rb; g.blk_off = 0; g.blk_cap = rb.cap; g.raster_band = kRasterBandFwd;
+    g.ids = ids; g.partials = partials; g.tgt = tgt; g.rows_cap = cap_rows; g.status = status_dev;
+    TRL_CUDA_OK(launch_tc_gemm(g, s));
+    launch_merge_lse(partials, tgt, nt, cap_rows, rb, ids, len, B, T, V, logp, lse, status_dev, s);
+  } else {
+    const size_t avail = workspace_bytes - row_blocks_bytes(B, T);
+    const int R = fit_rows(avail, cap_rows < kRecommendedChunkRowsF32 ? cap_rows : kRecommendedChunkRowsF32,
+                           [&](int r) { return align_up((size_t)r * H * 4, 256) + align_up((size_t)r * V * 4, 256); });
+    if (R < kRowBlock) return TRL_ERR_WORKSPACE_TOO_SMALL;
+    float* Xp = cv.take<float>((size_t)R * H);
+    float* S = cv.take<float>((size_t)R * V);
+    const int CB = R / kRowBlock;
+    launch_zero_padded_f32(logp, lse, len, B, T, s);
+    for (int blk_off = 0; blk_off < rb.cap; blk_off += CB) {
+      launch_pack_rows_f32((const float*)hidden, Xp, H, R, rb, blk_off, s);
+      SimtGemm sg{Xp, H, 1, (const float*)W, 1, H, S, V, R, V, H, 0, 1, rb.nblk, blk_off, CB};
+      launch_simt_gemm(sg, s);
+      launch_row_lse_f32(S, V, R, rb, blk_off, ids, logp, lse, status_dev, s);
+    }
+  }
+  TRL_CUDA_OK(cudaGetLastError());
+  return TRL_OK;
+}
+
+int trl_hrd_advantages(const float* r_plan, const float* r_code, const int32_t* len, const int32_t* bnd,
+                       int P, int G, int T, int adv_mode, float* A_plan, float* A_code, uint8_t* seg, float* adv,
+                       int32_t* n_plan, int32_t* n_code, int64_t* n_valid, int32_t* status_dev, void* stream) {
+  if (!r_plan || !r_code || !len || !bnd || !A_plan || !A_code || !seg || !adv || !n_plan || !n_code || !n_valid)
+    return TRL_ERR_INVALID_ARG;
+  if (P <= 0 || G <= 0 || T <= 0 || (long)P * G > 65535 || (long)P * G * T >= (1L << 31)) return TRL_ERR_SHAPE;
+  if (adv_mode != 0 && adv_mode != 1) return TRL_ERR_INVALID_ARG;
+  if (int e = check_device()) return e;
+  launch_hrd_advantages(r_plan, r_code, len, bnd, P, G, T, adv_mode, A_plan, A_code, seg, adv, n_plan, n_code,
+                        n_valid, status_dev, (cudaStream_t)stream);
+  TRL_CUDA_OK(cudaGetLastError());
+  return TRL_OK;
+}
+
+int trl_pg_loss_fwd(const float* logp, const float* old_logp, const float* adv, const uint8_t* seg,
+                    const int32_t* len, int P, int G, int T, trl_pg_config cfg, float* loss, float* g, float* stats,
+                    void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream) {
+  (void)status_dev;
+  if (!logp || !old_logp || !adv || !seg || !len || !loss || !g || !workspace) return TRL_ERR_INVALID_ARG;
+  if (P <= 0 || G <= 0 || T <= 0 || (long)P * G > 65535 || (long)P * G * T >= (1L << 31)) return TRL_ERR_SHAPE;
+  if (!(cfg.eps_lo >= 0.f) || !(cfg.eps_hi >= 0.f) || !(cfg.alpha >= 0.f)) return TRL_ERR_INVALID_ARG;
+  if (workspace_bytes < trl_workspace_bytes(TRL_CALL_PG_LOSS_FWD, P * G, T, 1, 1, TRL_F32)) return TRL_ERR_WORKSPACE_TOO_SMALL;
+  if (int e = check_device()) return e;
+  launch_pg_loss(logp, old_logp, adv, seg, len, P, G, T, cfg, loss, g, stats, (float*)workspace, (cudaStream_t)stream);
+  TRL_CUDA_OK(cudaGetLastError());
+  return TRL_OK;
+}
+
+int trl_pg_loss_bwd(const void* hidden, const void* W, const int32_t* ids, const int32_t* len, const float* lse,
+                    const float* g, int B, int T, int H, int V, trl_dtype dt, void* dHidden, float* dW,
+                    void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream) {
+  if (!hidden || !W || !ids || !len || !lse || !g || !dHidden || !dW || !workspace) return TRL_ERR_INVALID_ARG;
+  if (dt != TRL_F32 && dt != TRL_BF16) return TRL_ERR_DTYPE;
+  if (!shapes_ok(B, T, H, V)) return TRL_ERR_SHAPE;
+  if (dt == TRL_BF16 && ((H % 8) || (V % 8))) return TRL_ERR_SHAPE;
+  if (((uintptr_t)workspace & 255) != 0) return TRL_ERR_INVALID_ARG;
+  if (workspace_bytes < trl_workspace_bytes_min(TRL_CALL_PG_LOSS_BWD, B, T, H, V, dt)) return TRL_ERR_WORKSPACE_TOO_SMALL;
+  if (int e = check_device()) return e;
+  cudaStream_t s = (cudaStream_t)stream;
+  const int cap_rows = rows_cap_of(B, T);
+  const size_t N = (size_t)B * T;
+
+  Carver cv(workspace);
+  RowBlocks rb = carve_row_blocks(cv.take<char>(row_blocks_bytes(B, T)), B, T);
+  launch_build_row_blocks(len, B, T, rb, status_dev, s);
+  TRL_CUDA_OK(cudaMemsetAsync(dW, 0, (size_t)V * H * sizeof(float), s));
+
+  if (dt == TRL_BF16) {
+    TRL_CUDA_OK(cudaMemsetAsync(dHidden, 0, N * H * 2, s));
+    const size_t avail = workspace_bytes - bwd_fixed_bf16(B, T, H, V);
+    const int R = fit_rows(avail, cap_rows < kRecommendedChunkRowsBf16 ? cap_rows : kRecommendedChunkRowsBf16,
+                           [&](int r) { return bwd_per_rows_bf16(H, V, r); });
+    if (R < kRowBlock) return TRL_ERR_WORKSPACE_TOO_SMALL;
+    __nv_bfloat16* Wt = cv.take<__nv_bfloat16>((size_t)H * V);
+    __nv_bfloat16* Xt = cv.take<__nv_bfloat16>((size_t)H * R);
+    __nv_bfloat16* dS = cv.take<__nv_bfloat16>((size_t)R * V);
+    __nv_bfloat16* dSt = cv.take<__nv_bfloat16>((size_t)V * R);
+    launch_transpose_bf16((const __nv_bfloat16*)W, Wt, V, H, s);
+    const int CB = R / kRowBlock;
+    for (int blk_off = 0; blk_off < rb.cap; blk_off += CB) {
+      launch_gather_transpose_bf16((const __nv_bfloat16*)hidden, Xt, H, R, rb, blk_off, s);
+      TcGemm a;
+      memset(&a, 0, sizeof(a));
+      a.rb = rb; a.blk_off = blk_off; a.blk_cap = CB; a.status = status_dev;
+      // dS chunk = g (onehot - softmax), from a recomputed logits tile
+      TcGemm ds = a;
+      ds.epi = TC_EPI_DS; ds.raster_band = kRasterBandFwd;
+      ds.A = hidden; ds.a_rows = (long)N; ds.a_ld = H; ds.B = W; ds.b_rows = V; ds.b_ld = H; ds.K = H; ds.N = V;
+      ds.ids = ids; ds.lse = lse; ds.g = g; ds.dS = dS; ds.ds_ld = V; ds.dSt = dSt; ds.dst_ld = R;
+      TRL_CUDA_OK(launch_tc_gemm(ds, s));
+      // dHidden rows of the chunk = dS W
+      TcGemm dh = a;
+      dh.epi = TC_EPI_DH; dh.raster_band = kRasterBandBwd;
+      dh.A = dS; dh.a_rows = R; dh.a_ld = V; dh.B = Wt; dh.b_rows = H; dh.b_ld = V; dh.K = V; dh.N = H;
+      dh.dHidden = (__nv_bfloat16*)dHidden; dh.dh_ld = H;
+      TRL_CUDA_OK(launch_tc_gemm(dh, s));
+      // dW += dS^T hidden
+      TcGemm dw = a;
+      dw.epi = TC_EPI_DW; dw.raster_band = kRasterBandBwd;
+      dw.A = dSt; dw.a_rows = V; dw.a_ld = R; dw.B = Xt; dw.b_rows = H; dw.b_ld = R; dw.K = R; dw.N = H;
+      dw.m_blocks = cdiv(V, kRowBlock); dw.dW = dW; dw.dw_ld = H; dw.V = V;
+      TRL_CUDA_OK(launch_tc_gemm(dw, s));
+    }
+  } else {
+    TRL_CUDA_OK(cudaMemsetAsync(dHidden, 0, N * H * 4, s));
+    const size_t avail = workspace_bytes - row_blocks_bytes(B, T);
+    const int R = fit_rows(avail, cap_rows < kRecommendedChunkRowsF32 ? cap_rows : kRecommendedChunkRowsF32,
+                           [&](int r) { return 2 * align_up((size_t)r * H * 4, 256) + align_up((size_t)r * V * 4, 256); });
+    if (R < kRowBlock) return TRL_ERR_WORKSPACE_TOO_SMALL;
+    float* Xp = cv.take<float>((size_t)R * H);
+    float* dHp = cv.take<float>((size_t)R * H);
+    float* S = cv.take<float>((size_t)R * V);
+    const int CB = R / kRowBlock;
+    for (int blk_off = 0; blk_off < rb.cap; blk_off += CB) {
+      launch_pack_rows_f32((const float*)hidden, Xp, H, R, rb, blk_off, s);
+      SimtGemm fwd{Xp, H, 1, (const float*)W, 1, H, S, V, R, V, H, 0, 1, rb.nblk, blk_off, CB};
+      launch_simt_gemm(fwd, s);
+      launch_ds_inplace_f32(S, V, R, rb, blk_off, ids, lse, g, s);
+      SimtGemm dh{S, V, 1, (const float*)W, H, 1, dHp, H, R, H, V, 0, 1, rb.nblk, blk_off, CB};
+      launch_simt_gemm(dh, s);
+      launch_scatter_rows_f32(dHp, (float*)dHidden, H, R, rb, blk_off, s);
+      SimtGemm dw{S, 1, V, Xp, H, 1, dW, H, V, H, R, 1, 2, rb.nblk, blk_off, CB};
+      launch_simt_gemm(dw, s);
+    }
+  }
+  TRL_CUDA_OK(cudaGetLastError());
+  return TRL_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,94 @@
+// Internal declarations shared by the translation units of libtrl (host side only).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "trl.h"
+
+namespace trl {
+
+constexpr int kRowBlock = 128;   // rows per row block = TMEM lanes of one accumulator tile
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+inline int cdiv(int a, int b) { return (a + b - 1) / b; }
+
+// Row blocks: every rollout's valid rows [b*T, b*T+len) are cut into blocks of <=128
+// consecutive rows.  Built on the device from `len` (no host round trip).
+struct RowBlocks {
+  int* nblk;       // [1]   number of live blocks
+  int* blk_first;  // [B+1] first block of each rollout (exclusive prefix sum)
+  int* blk_row;    // [cap] global row index of the block's first row
+  int* blk_n;      // [cap] valid rows in the block (1..128)
+  int cap;         // B * ceil(T/128): upper bound on nblk
+};
+size_t row_blocks_bytes(int B, int T);
+RowBlocks carve_row_blocks(void* base, int B, int T);
+
+// ---- small kernels (trl_small_kernels.cu) ------------------------------------------
+void launch_build_row_blocks(const int32_t* len, int B, int T, RowBlocks rb, int32_t* status, cudaStream_t s);
+void launch_hrd_advantages(const float* r_plan, const float* r_code, const int32_t* len, const int32_t* bnd,
+                           int P, int G, int T, int adv_mode, float* A_plan, float* A_code, uint8_t* seg,
+                           float* adv, int32_t* n_plan, int32_t* n_code, int64_t* n_valid, int32_t* status,
+                           cudaStream_t s);
+int  pg_loss_tiles(int T);
+void launch_pg_loss(const float* logp, const float* old_logp, const float* adv, const uint8_t* seg,
+                    const int32_t* len, int P, int G, int T, trl_pg_config cfg, float* loss, float* g,
+                    float* stats, float* partials, cudaStream_t s);
+// merge per-vocabulary-tile (max, sumexp) partials into lse / logp and scatter to global rows
+void launch_merge_lse(const float2* partials, const float* tgt, int n_tiles, int rows_cap, RowBlocks rb,
+                      const int32_t* ids, const int32_t* len, int B, int T, int V, float* logp, float* lse,
+                      int32_t* status, cudaStream_t s);
+void launch_transpose_bf16(const __nv_bfloat16* in, __nv_bfloat16* out, int rows, int cols, cudaStream_t s);
+// Xt[h, r] = hidden[row(blk_off*128 + r), h] for the live rows of a chunk, 0 elsewhere
+void launch_gather_transpose_bf16(const __nv_bfloat16* hidden, __nv_bfloat16* Xt, int H, int R, RowBlocks rb,
+                                  int blk_off, cudaStream_t s);
+// fp32 path helpers
+void launch_pack_rows_f32(const float* hidden, float* Xp, int H, int R, RowBlocks rb, int blk_off, cudaStream_t s);
+void launch_row_lse_f32(const float* S, int V, int R, RowBlocks rb, int blk_off, const int32_t* ids,
+                        float* logp, float* lse, int32_t* status, cudaStream_t s);
+void launch_ds_inplace_f32(float* S, int V, int R, RowBlocks rb, int blk_off, const int32_t* ids,
+                           const float* lse, const float* g, cudaStream_t s);
+void launch_scatter_rows_f32(const float* dHp, float* dHidden, int H, int R, RowBlocks rb, int blk_off, cudaStream_t s);
+void launch_zero_padded_f32(float* a, float* b, const int32_t* len, int B, int T, cudaStream_t s);
+
+// ---- fp32 CUDA-core GEMM (trl_simt_gemm.cu) ----------------------------------------
+// C[m,n] (+)= sum_k A(m,k) B(k,n); A(m,k) = A[m*sam + k*sak], B(k,n) = B[k*sbk + n*sbn].
+// If live_from_blocks != 0 the extent named by it (1: M, 2: K) is
+// 128 * clamp(*nblk - blk_off, 0, blk_cap) instead of the host value.
+struct SimtGemm {
+  const float* A; long sam, sak;
+  const float* B; long sbk, sbn;
+  float* C; long ldc;
+  int M, N, K;
+  int accumulate;
+  int live_from_blocks; const int* nblk; int blk_off, blk_cap;
+};
+void launch_simt_gemm(const SimtGemm& p, cudaStream_t s);
+
+// ---- tcgen05 GEMM family (trl_tc_gemm.cu) ------------------------------------------
+enum TcEpilogue { TC_EPI_LSE = 0, TC_EPI_DS = 1, TC_EPI_DH = 2, TC_EPI_DW = 3 };
+struct TcGemm {
+  int epi;
+  // operands: A [a_rows, K] and B [b_rows, K], both bf16 row-major with K contiguous
+  const void* A; long a_rows; long a_ld;     // a_ld = row pitch in elements
+  const void* B; long b_rows; long b_ld;
+  int K;                                     // host K extent (TC_EPI_DW: K = 128 * live blocks of the chunk)
+  int N;                                     // GEMM N extent = b_rows that are meaningful
+  int m_blocks;                              // TC_EPI_DW: fixed number of 128-row blocks of A; others: from row blocks
+  RowBlocks rb; int blk_off, blk_cap;        // chunk of row blocks
+  int raster_band;
+  // epilogue arguments
+  const int32_t* ids; const float* lse; const float* g;
+  float2* partials; float* tgt; int rows_cap;          // LSE
+  __nv_bfloat16* dS; long ds_ld; __nv_bfloat16* dSt; long dst_ld;   // DS
+  __nv_bfloat16* dHidden; long dh_ld;                  // DH
+  float* dW; long dw_ld; int V;                        // DW
+  int32_t* status;
+};
+// returns cudaSuccess or the error of tensor-map creation / launch
+cudaError_t launch_tc_gemm(const TcGemm& p, cudaStream_t s);
+int tc_num_sms();
+
+}  // namespace trl

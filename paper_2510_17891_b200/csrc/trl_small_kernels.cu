@@ -1,0 +1,461 @@
+// Memory-bound kernels of the HRD policy-gradient path: row-block construction, HRD
+// advantages (Section 2.3, Eq. 2), the clipped surrogate and its derivative, the merge of
+// per-vocabulary-tile log-sum-exp partials, and layout helpers.
+#include "trl_internal.h"
+
+namespace trl {
+
+__device__ __forceinline__ void flag_status(int32_t* status, int code) {
+  if (status) atomicOr(status, 1 << code);
+}
+
+size_t row_blocks_bytes(int B, int T) {
+  size_t cap = (size_t)B * cdiv(T, kRowBlock);
+  return align_up((1 + (size_t)B + 1 + 2 * cap) * sizeof(int), 256);
+}
+
+RowBlocks carve_row_blocks(void* base, int B, int T) {
+  RowBlocks rb;
+  int* p = (int*)base;
+  rb.cap = B * cdiv(T, kRowBlock);
+  rb.nblk = p;
+  rb.blk_first = p + 1;
+  rb.blk_row = p + 1 + (B + 1);
+  rb.blk_n = rb.blk_row + rb.cap;
+  return rb;
+}
+
+// One CTA.  Pass 1: per-thread serial counts over a contiguous slice of rollouts, block
+// scan over slices; pass 2: each rollout writes its blocks.
+__global__ void build_row_blocks_kernel(const int32_t* __restrict__ len, int B, int T, RowBlocks rb,
+                                        int32_t* status) {
+  __shared__ int s_sum[1024];
+  const int tid = threadIdx.x, nt = blockDim.x;
+  const int per = (B + nt - 1) / nt;
+  const int b0 = min(tid * per, B), b1 = min(b0 + per, B);
+  int cnt = 0;
+  bool bad = false;
+  for (int b = b0; b < b1; ++b) {
+    int L = len[b];
+    if (L < 0 || L > T) { bad = true; L = max(0, min(L, T)); }
+    cnt += (L + kRowBlock - 1) / kRowBlock;
+  }
+  if (bad) flag_status(status, TRL_ERR_BAD_INDEX);
+  s_sum[tid] = cnt;
+  __syncthreads();
+  // inclusive Hillis-Steele scan
+  for (int off = 1; off < nt; off <<= 1) {
+    int v = (tid >= off) ? s_sum[tid - off] : 0;
+    __syncthreads();
+    s_sum[tid] += v;
+    __syncthreads();
+  }
+  int first = s_sum[tid] - cnt;
+  if (tid == nt - 1) { rb.nblk[0] = s_sum[tid]; rb.blk_first[B] = s_sum[tid]; }
+  for (int b = b0; b < b1; ++b) {
+    int L = max(0, min(len[b], T));
+    rb.blk_first[b] = first;
+    int nb = (L + kRowBlock - 1) / kRowBlock;
+    for (int i = 0; i < nb; ++i) {
+      rb.blk_row[first + i] = b * T + i * kRowBlock;
+      rb.blk_n[first + i] = min(kRowBlock, L - i * kRowBlock);
+    }
+    first += nb;
+  }
+}
+
+void launch_build_row_blocks(const int32_t* len, int B, int T, RowBlocks rb, int32_t* status, cudaStream_t s) {
+  build_row_blocks_kernel<<<1, 1024, 0, s>>>(len, B, T, rb, status);
+}
+
+// ------------------------------------------------------------------------------------
+// HRD advantages.  grid = (token tiles, B).  Each CTA re-derives its group's means with a
+// warp-shuffle reduction over the G rewards of the prompt (fp64), then streams out the
+// segment labels and per-token advantages of its token tile with 16-byte stores.
+// ------------------------------------------------------------------------------------
+constexpr int kAdvTile = 8192;   // tokens per CTA
+
+__device__ __forceinline__ double warp_sum(double v) {
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+__global__ void __launch_bounds__(256) hrd_adv_kernel(
+    const float* __restrict__ r_plan, const float* __restrict__ r_code, const int32_t* __restrict__ len,
+    const int32_t* __restrict__ bnd, int P, int G, int T, int adv_mode, float* __restrict__ A_plan,
+    float* __restrict__ A_code, uint8_t* __restrict__ seg, float* __restrict__ adv, int32_t* __restrict__ n_plan,
+    int32_t* __restrict__ n_code, int64_t* __restrict__ n_valid, int32_t* status) {
+  __shared__ float s_A[2];
+  __shared__ int s_lb[2];
+  const int b = blockIdx.y, i = b / G;
+  const int tid = threadIdx.x;
+  if (tid < 32) {
+    double sp = 0, sc = 0;
+    for (int j = tid; j < G; j += 32) { sp += (double)r_plan[i * G + j]; sc += (double)r_code[i * G + j]; }
+    sp = warp_sum(sp); sc = warp_sum(sc);
+    const double mp = sp / G, mc = sc / G;
+    double ap = (double)r_plan[b] - mp, ac = (double)r_code[b] - mc;
+    if (adv_mode == 1) {
+      double vp = 0, vc = 0;
+      for (int j = tid; j < G; j += 32) {
+        double dp = (double)r_plan[i * G + j] - mp, dc = (double)r_code[i * G + j] - mc;
+        vp += dp * dp; vc += dc * dc;
+      }
+      vp = warp_sum(vp); vc = warp_sum(vc);
+      ap /= (sqrt(vp / G) + 1e-6); ac /= (sqrt(vc / G) + 1e-6);
+    }
+    if (tid == 0) {
+      int L = len[b], Bd = bnd[b];
+      bool bad = (L < 0 || L > T);
+      L = max(0, min(L, T));
+      bad |= (Bd < 0 || Bd > L);
+      Bd = max(0, min(Bd, L));
+      if (bad) flag_status(status, TRL_ERR_BAD_INDEX);
+      s_A[0] = (float)ap; s_A[1] = (float)ac; s_lb[0] = L; s_lb[1] = Bd;
+      if (blockIdx.x == 0) {
+        A_plan[b] = (float)ap; A_code[b] = (float)ac; n_plan[b] = Bd; n_code[b] = L - Bd;
+      }
+    }
+    if (blockIdx.x == 0 && b == 0) {          // sum of lengths: one warp, fixed order, integers
+      long long tot = 0;
+      for (int k = tid; k < P * G; k += 32) tot += max(0, min(len[k], T));
+      for (int o = 16; o > 0; o >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, o);
+      if (tid == 0) n_valid[0] = tot;
+    }
+  }
+  __syncthreads();
+  const float ap = s_A[0], ac = s_A[1];
+  const int L = s_lb[0], Bd = s_lb[1];
+  const int t_begin = blockIdx.x * kAdvTile, t_end = min(T, t_begin + kAdvTile);
+  const size_t base = (size_t)b * T;
+  // 16 tokens per thread-iteration when the row start is 16-aligned, else scalar
+  if ((T & 15) == 0) {
+    for (int t = t_begin + tid * 16; t < t_end; t += 256 * 16) {
+      uint32_t w[4];
+      float a[16];
+#pragma unroll
+      for (int q = 0; q < 16; ++q) {
+        const int tt = t + q;
+        const int sg = tt < Bd ? 1 : (tt < L ? 2 : 0);
+        a[q] = sg == 1 ? ap : (sg == 2 ? ac : 0.f);
+        if ((q & 3) == 0) w[q >> 2] = 0;
+        w[q >> 2] |= (uint32_t)sg << (8 * (q & 3));
+      }
+      *reinterpret_cast<uint4*>(seg + base + t) = make_uint4(w[0], w[1], w[2], w[3]);
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        *reinterpret_cast<float4*>(adv + base + t + 4 * q) = make_float4(a[4 * q], a[4 * q + 1], a[4 * q + 2], a[4 * q + 3]);
+    }
+  } else {
+    for (int t = t_begin + tid; t < t_end; t += 256) {
+      const int sg = t < Bd ? 1 : (t < L ? 2 : 0);
+      seg[base + t] = (uint8_t)sg;
+      adv[base + t] = sg == 1 ? ap : (sg == 2 ? ac : 0.f);
+    }
+  }
+}
+
+void launch_hrd_advantages(const float* r_plan, const float* r_code, const int32_t* len, const int32_t* bnd,
+                           int P, int G, int T, int adv_mode, float* A_plan, float* A_code, uint8_t* seg,
+                           float* adv, int32_t* n_plan, int32_t* n_code, int64_t* n_valid, int32_t* status,
+                           cudaStream_t s) {
+  dim3 grid(cdiv(T, kAdvTile), P * G);
+  hrd_adv_kernel<<<grid, 256, 0, s>>>(r_plan, r_code, len, bnd, P, G, T, adv_mode, A_plan, A_code, seg, adv,
+                                      n_plan, n_code, n_valid, status);
+}
+
+// ------------------------------------------------------------------------------------
+// Clipped surrogate.  Stage 1: grid = (tiles, B), each CTA reduces its token tile of one
+// rollout in a fixed order and writes 4 partial sums; also writes g.  Stage 2: one CTA
+// combines the partials in index order in fp64 -> bit-reproducible loss.
+// ------------------------------------------------------------------------------------
+constexpr int kLossTile = 4096;
+int pg_loss_tiles(int T) { return cdiv(T, kLossTile); }
+
+__global__ void __launch_bounds__(256) pg_loss_stage1_kernel(
+    const float* __restrict__ logp, const float* __restrict__ old_logp, const float* __restrict__ adv,
+    const uint8_t* __restrict__ seg, const int32_t* __restrict__ len, int P, int G, int T, trl_pg_config cfg,
+    float* __restrict__ g, float* __restrict__ partials) {
+  const int b = blockIdx.y, tid = threadIdx.x;
+  const int L = max(0, min(len[b], T));
+  const int t_begin = blockIdx.x * kLossTile, t_end = min(T, t_begin + kLossTile);
+  const size_t base = (size_t)b * T;
+  const float inv = L > 0 ? 1.0f / ((float)P * (float)G * (float)L) : 0.f;
+  const float lo = 1.0f - cfg.eps_lo, hi = 1.0f + cfg.eps_hi;
+  float acc = 0.f, n_hi = 0.f, n_lo = 0.f, sum_s = 0.f;
+  for (int t = t_begin + tid; t < t_end; t += 256) {
+    float gn = 0.f;
+    if (t < L) {
+      const size_t n = base + t;
+      const float s = expf(logp[n] - old_logp[n]);
+      const float A = adv[n];
+      const int sg = seg[n];
+      const float w = sg == 1 ? cfg.alpha : (sg == 2 ? 1.0f : 0.f);
+      const float unclipped = A * s;
+      const float clipped = A * fminf(fmaxf(s, lo), hi);
+      acc += w * fminf(unclipped, clipped);
+      if (unclipped <= clipped) gn = -w * A * s * inv;
+      n_hi += s > hi ? 1.f : 0.f;
+      n_lo += s < lo ? 1.f : 0.f;
+      sum_s += s;
+    }
+    g[base + t] = gn;
+  }
+  __shared__ float red[4][8];
+  float v[4] = {acc, n_hi, n_lo, sum_s};
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    for (int o = 16; o > 0; o >>= 1) v[q] += __shfl_xor_sync(0xffffffffu, v[q], o);
+    if ((tid & 31) == 0) red[q][tid >> 5] = v[q];
+  }
+  __syncthreads();
+  if (tid < 4) {
+    float s = 0.f;
+    for (int w = 0; w < 8; ++w) s += red[tid][w];
+    partials[((size_t)b * gridDim.x + blockIdx.x) * 4 + tid] = s;
+  }
+}
+
+__global__ void __launch_bounds__(256) pg_loss_stage2_kernel(const float* __restrict__ partials,
+                                                             const int32_t* __restrict__ len, int P, int G, int T,
+                                                             int tiles, float* __restrict__ loss,
+                                                             float* __restrict__ stats) {
+  __shared__ double red[4][256];
+  const int tid = threadIdx.x, B = P * G;
+  double J = 0, nh = 0, nl = 0, ss = 0;
+  for (int b = tid; b < B; b += 256) {
+    const int L = max(0, min(len[b], T));
+    double a = 0;
+    for (int k = 0; k < tiles; ++k) {
+      const float* p = partials + ((size_t)b * tiles + k) * 4;
+      a += p[0]; nh += p[1]; nl += p[2]; ss += p[3];
+    }
+    if (L > 0) J += a / L;
+  }
+  red[0][tid] = J; red[1][tid] = nh; red[2][tid] = nl; red[3][tid] = ss;
+  __syncthreads();
+  if (tid == 0) {
+    double t[4] = {0, 0, 0, 0};
+    for (int q = 0; q < 4; ++q)
+      for (int k = 0; k < 256; ++k) t[q] += red[q][k];
+    long long ntok = 0;
+    for (int b = 0; b < B; ++b) ntok += max(0, min(len[b], T));
+    loss[0] = (float)(-t[0] / ((double)P * (double)G));
+    if (stats) {
+      const double d = ntok > 0 ? (double)ntok : 1.0;
+      stats[0] = (float)(t[1] / d); stats[1] = (float)(t[2] / d); stats[2] = (float)(t[3] / d);
+      stats[3] = (float)ntok;
+    }
+  }
+}
+
+void launch_pg_loss(const float* logp, const float* old_logp, const float* adv, const uint8_t* seg,
+                    const int32_t* len, int P, int G, int T, trl_pg_config cfg, float* loss, float* g,
+                    float* stats, float* partials, cudaStream_t s) {
+  const int tiles = pg_loss_tiles(T);
+  dim3 grid(tiles, P * G);
+  pg_loss_stage1_kernel<<<grid, 256, 0, s>>>(logp, old_logp, adv, seg, len, P, G, T, cfg, g, partials);
+  pg_loss_stage2_kernel<<<1, 256, 0, s>>>(partials, len, P, G, T, tiles, loss, stats);
+}
+
+// ------------------------------------------------------------------------------------
+// Merge of per-vocabulary-tile partials: lse = M + log sum_k l_k exp(m_k - M).
+// One thread per global row; padded rows get 0.
+// ------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) merge_lse_kernel(const float2* __restrict__ partials,
+                                                        const float* __restrict__ tgt, int n_tiles, int rows_cap,
+                                                        RowBlocks rb, const int32_t* __restrict__ ids,
+                                                        const int32_t* __restrict__ len, int B, int T, int V,
+                                                        float* __restrict__ logp, float* __restrict__ lse,
+                                                        int32_t* status) {
+  const size_t n = (size_t)blockIdx.x * 256 + threadIdx.x;
+  if (n >= (size_t)B * T) return;
+  const int b = (int)(n / T), t = (int)(n % T);
+  const int L = max(0, min(len[b], T));
+  float out_lp = 0.f, out_lse = 0.f;
+  if (t < L) {
+    const size_t prow = (size_t)(rb.blk_first[b] + t / kRowBlock) * kRowBlock + (t % kRowBlock);
+    float M = -INFINITY;
+    for (int k = 0; k < n_tiles; ++k) M = fmaxf(M, partials[(size_t)k * rows_cap + prow].x);
+    float l = 0.f;
+    for (int k = 0; k < n_tiles; ++k) {
+      const float2 p = partials[(size_t)k * rows_cap + prow];
+      l += p.y * __expf(p.x - M);
+    }
+    out_lse = M + __logf(l);
+    const int id = ids[n];
+    if ((unsigned)id < (unsigned)V) out_lp = tgt[prow] - out_lse;
+    else flag_status(status, TRL_ERR_BAD_INDEX);
+  }
+  logp[n] = out_lp;
+  lse[n] = out_lse;
+}
+
+void launch_merge_lse(const float2* partials, const float* tgt, int n_tiles, int rows_cap, RowBlocks rb,
+                      const int32_t* ids, const int32_t* len, int B, int T, int V, float* logp, float* lse,
+                      int32_t* status, cudaStream_t s) {
+  const size_t N = (size_t)B * T;
+  merge_lse_kernel<<<(unsigned)((N + 255) / 256), 256, 0, s>>>(partials, tgt, n_tiles, rows_cap, rb, ids, len, B, T,
+                                                               V, logp, lse, status);
+}
+
+// ------------------------------------------------------------------------------------
+// bf16 transposes (64x64 tiles through shared memory)
+// ------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) transpose_bf16_kernel(const __nv_bfloat16* __restrict__ in,
+                                                             __nv_bfloat16* __restrict__ out, int rows, int cols) {
+  __shared__ __nv_bfloat16 tile[64][66];
+  const int r0 = blockIdx.y * 64, c0 = blockIdx.x * 64;
+  const int tx = threadIdx.x & 63, ty = threadIdx.x >> 6;
+  for (int i = ty; i < 64; i += 4) {
+    const int r = r0 + i, c = c0 + tx;
+    tile[i][tx] = (r < rows && c < cols) ? in[(size_t)r * cols + c] : __float2bfloat16(0.f);
+  }
+  __syncthreads();
+  for (int i = ty; i < 64; i += 4) {
+    const int c = c0 + i, r = r0 + tx;
+    if (c < cols && r < rows) out[(size_t)c * rows + r] = tile[tx][i];
+  }
+}
+
+void launch_transpose_bf16(const __nv_bfloat16* in, __nv_bfloat16* out, int rows, int cols, cudaStream_t s) {
+  dim3 grid(cdiv(cols, 64), cdiv(rows, 64));
+  transpose_bf16_kernel<<<grid, 256, 0, s>>>(in, out, rows, cols);
+}
+
+// Xt [H, R]: column r is hidden row (block blk_off + r/128, lane r%128) or 0 if not live.
+__global__ void __launch_bounds__(256) gather_transpose_bf16_kernel(const __nv_bfloat16* __restrict__ hidden,
+                                                                    __nv_bfloat16* __restrict__ Xt, int H, int R,
+                                                                    RowBlocks rb, int blk_off) {
+  __shared__ __nv_bfloat16 tile[64][66];
+  const int r0 = blockIdx.y * 64, h0 = blockIdx.x * 64;     // r0: scratch row, 64 | 128 so one block per tile
+  const int blk = blk_off + r0 / kRowBlock;
+  const int live = blk < rb.nblk[0];
+  const int tx = threadIdx.x & 63, ty = threadIdx.x >> 6;
+  const long grow0 = live ? (long)rb.blk_row[blk] : 0;
+  const int nvalid = live ? rb.blk_n[blk] : 0;
+  for (int i = ty; i < 64; i += 4) {
+    const int lr = (r0 % kRowBlock) + i;
+    const int h = h0 + tx;
+    tile[i][tx] = (lr < nvalid && h < H) ? hidden[(size_t)(grow0 + lr) * H + h] : __float2bfloat16(0.f);
+  }
+  __syncthreads();
+  for (int i = ty; i < 64; i += 4) {
+    const int h = h0 + i, r = r0 + tx;
+    if (h < H && r < R) Xt[(size_t)h * R + r] = tile[tx][i];
+  }
+}
+
+void launch_gather_transpose_bf16(const __nv_bfloat16* hidden, __nv_bfloat16* Xt, int H, int R, RowBlocks rb,
+                                  int blk_off, cudaStream_t s) {
+  dim3 grid(cdiv(H, 64), cdiv(R, 64));
+  gather_transpose_bf16_kernel<<<grid, 256, 0, s>>>(hidden, Xt, H, R, rb, blk_off);
+}
+
+// ------------------------------------------------------------------------------------
+// fp32 path helpers.  Scratch row r of a chunk is (block blk_off + r/128, lane r%128).
+// ------------------------------------------------------------------------------------
+__device__ __forceinline__ long scratch_row_to_global(const RowBlocks& rb, int blk_off, int r) {
+  const int blk = blk_off + r / kRowBlock;
+  if (blk >= rb.nblk[0]) return -1;
+  const int lr = r % kRowBlock;
+  return lr < rb.blk_n[blk] ? (long)rb.blk_row[blk] + lr : -1;
+}
+
+__global__ void pack_rows_f32_kernel(const float* __restrict__ hidden, float* __restrict__ Xp, int H, int R,
+                                     RowBlocks rb, int blk_off) {
+  const int r = blockIdx.x;
+  const long n = scratch_row_to_global(rb, blk_off, r);
+  for (int h = threadIdx.x; h < H; h += blockDim.x) Xp[(size_t)r * H + h] = n >= 0 ? hidden[(size_t)n * H + h] : 0.f;
+}
+void launch_pack_rows_f32(const float* hidden, float* Xp, int H, int R, RowBlocks rb, int blk_off, cudaStream_t s) {
+  pack_rows_f32_kernel<<<R, 128, 0, s>>>(hidden, Xp, H, R, rb, blk_off);
+}
+
+__device__ __forceinline__ float block_reduce(float v, bool is_max, float* sh) {
+  for (int o = 16; o > 0; o >>= 1) {
+    float u = __shfl_xor_sync(0xffffffffu, v, o);
+    v = is_max ? fmaxf(v, u) : v + u;
+  }
+  const int w = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) sh[w] = v;
+  __syncthreads();
+  float r = sh[0];
+  for (int k = 1; k < nw; ++k) r = is_max ? fmaxf(r, sh[k]) : r + sh[k];
+  return r;
+}
+
+__global__ void __launch_bounds__(256) row_lse_f32_kernel(const float* __restrict__ S, int V, int R, RowBlocks rb,
+                                                          int blk_off, const int32_t* __restrict__ ids,
+                                                          float* __restrict__ logp, float* __restrict__ lse,
+                                                          int32_t* status) {
+  __shared__ float sh[8];
+  const int r = blockIdx.x;
+  const long n = scratch_row_to_global(rb, blk_off, r);
+  if (n < 0) return;
+  const float* row = S + (size_t)r * V;
+  float m = -INFINITY;
+  for (int v = threadIdx.x; v < V; v += 256) m = fmaxf(m, row[v]);
+  m = block_reduce(m, true, sh);
+  float l = 0.f;
+  for (int v = threadIdx.x; v < V; v += 256) l += expf(row[v] - m);
+  l = block_reduce(l, false, sh);
+  if (threadIdx.x == 0) {
+    const float L = m + logf(l);
+    lse[n] = L;
+    const int id = ids[n];
+    if ((unsigned)id < (unsigned)V) logp[n] = row[id] - L;
+    else { logp[n] = 0.f; flag_status(status, TRL_ERR_BAD_INDEX); }
+  }
+}
+void launch_row_lse_f32(const float* S, int V, int R, RowBlocks rb, int blk_off, const int32_t* ids, float* logp,
+                        float* lse, int32_t* status, cudaStream_t s) {
+  row_lse_f32_kernel<<<R, 256, 0, s>>>(S, V, R, rb, blk_off, ids, logp, lse, status);
+}
+
+__global__ void __launch_bounds__(256) ds_inplace_f32_kernel(float* __restrict__ S, int V, int R, RowBlocks rb,
+                                                             int blk_off, const int32_t* __restrict__ ids,
+                                                             const float* __restrict__ lse,
+                                                             const float* __restrict__ g) {
+  const int r = blockIdx.x;
+  const long n = scratch_row_to_global(rb, blk_off, r);
+  float* row = S + (size_t)r * V;
+  if (n < 0) {
+    for (int v = threadIdx.x; v < V; v += 256) row[v] = 0.f;
+    return;
+  }
+  const float gn = g[n], L = lse[n];
+  const int id = ids[n];
+  for (int v = threadIdx.x; v < V; v += 256) row[v] = gn * ((v == id ? 1.f : 0.f) - expf(row[v] - L));
+}
+void launch_ds_inplace_f32(float* S, int V, int R, RowBlocks rb, int blk_off, const int32_t* ids, const float* lse,
+                           const float* g, cudaStream_t s) {
+  ds_inplace_f32_kernel<<<R, 256, 0, s>>>(S, V, R, rb, blk_off, ids, lse, g);
+}
+
+__global__ void scatter_rows_f32_kernel(const float* __restrict__ dHp, float* __restrict__ dHidden, int H, int R,
+                                        RowBlocks rb, int blk_off) {
+  const int r = blockIdx.x;
+  const long n = scratch_row_to_global(rb, blk_off, r);
+  if (n < 0) return;
+  for (int h = threadIdx.x; h < H; h += blockDim.x) dHidden[(size_t)n * H + h] = dHp[(size_t)r * H + h];
+}
+void launch_scatter_rows_f32(const float* dHp, float* dHidden, int H, int R, RowBlocks rb, int blk_off,
+                             cudaStream_t s) {
+  scatter_rows_f32_kernel<<<R, 128, 0, s>>>(dHp, dHidden, H, R, rb, blk_off);
+}
+
+__global__ void zero_padded_f32_kernel(float* __restrict__ a, float* __restrict__ b, const int32_t* __restrict__ len,
+                                       int B, int T) {
+  const size_t n = (size_t)blockIdx.x * 256 + threadIdx.x;
+  if (n >= (size_t)B * T) return;
+  const int bb = (int)(n / T), t = (int)(n % T);
+  if (t >= max(0, min(len[bb], T))) { a[n] = 0.f; b[n] = 0.f; }
+}
+void launch_zero_padded_f32(float* a, float* b, const int32_t* len, int B, int T, cudaStream_t s) {
+  const size_t N = (size_t)B * T;
+  zero_padded_f32_kernel<<<(unsigned)((N + 255) / 256), 256, 0, s>>>(a, b, len, B, T);
+}
+
+}  // namespace trl

@@ -1,0 +1,496 @@
+// tcgen05 / TMEM bf16 GEMM family for sm_100a.
+//
+// One persistent, warp-specialised kernel computes C[m,n] = sum_k A[m,k] B[n,k] (both
+// operands K-contiguous bf16, fp32 accumulation in tensor memory) on 128x256 tiles and
+// applies one of four epilogues straight from TMEM:
+//   LSE : per-row (max, sum-exp) of the tile's logits + pick-up of the sampled token's
+//         logit                                       (token scoring, Section 2.3 ratio s)
+//   DS  : dS = g (onehot - exp(z - lse)) as bf16, written row-major and transposed
+//   DH  : dHidden rows (bf16), scattered to the caller's row positions
+//   DW  : dW += tile (fp32 read-modify-write)
+//
+// Roles: warp 0 = TMA producer (one elected lane), warp 1 = MMA issuer (one elected lane)
+// and TMEM owner, warps 2..5 = epilogue (one TMEM lane quadrant each).  Shared-memory
+// stages are guarded by full/empty mbarriers; the 512 TMEM columns hold two 128x256 fp32
+// accumulators so the epilogue of tile i overlaps the mainloop of tile i+1.
+// Every wait is bounded: on expiry the CTA raises TRL_ERR_TIMEOUT in the status word,
+// all roles leave their loops, TMEM is freed and the kernel returns.
+#include <cuda.h>
+
+#include "trl_internal.h"
+
+namespace trl {
+
+namespace {
+
+constexpr int BM = 128, BN = 256, BK = 64, UMMA_K = 16, STAGES = 4;
+constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int NUM_THREADS = 192;
+constexpr uint32_t TMEM_COLS = 512;
+constexpr float LOG2E = 1.4426950408889634f, LN2 = 0.6931471805599453f;
+constexpr long long WAIT_CYCLES = 4000000000LL;   // ~2-3 s at B200 clocks
+
+struct TcArgs {
+  int N, K, m_blocks_fixed, blk_off, blk_cap, raster_band, rows_cap, V;
+  const int* nblk; const int* blk_row; const int* blk_n;
+  const int32_t* ids; const float* lse; const float* g;
+  float2* partials; float* tgt;
+  __nv_bfloat16* dS; long ds_ld; __nv_bfloat16* dSt; long dst_ld;
+  __nv_bfloat16* dHidden; long dh_ld;
+  float* dW; long dw_ld;
+  int32_t* status;
+};
+
+// ---------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok;
+}
+// Bounded wait.  Returns false if the CTA is aborting (own timeout or another role's).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  uint32_t spins = 0;
+  while (!mbar_try_wait(bar, parity)) {
+    if ((++spins & 255u) == 0) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > WAIT_CYCLES) {
+        *abort_flag = 1;
+        if (status) atomicOr(status, 1 << TRL_ERR_TIMEOUT);
+        return false;
+      }
+    }
+  }
+  return true;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(tm), "r"(bar), "r"(x), "r"(y)
+      : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
+                                            uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+        "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+        "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// Shared-memory matrix descriptor, K-major operand, 128-byte swizzle: rows are 128 B
+// apart inside an 8-row group, groups are 1024 B apart (stride byte offset); the leading
+// byte offset is not used for swizzled K-major layouts (set to 1); descriptor version 1.
+__device__ __forceinline__ uint64_t make_kmajor_sw128_desc(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr >> 4) & 0x3FFF);
+  d |= (uint64_t)1 << 16;
+  d |= (uint64_t)(1024 >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+// Instruction descriptor, kind::f16: D = fp32, A = B = bf16, both K-major, M x N tile.
+__host__ __device__ constexpr uint32_t make_idesc_bf16(int M, int N) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+__device__ __forceinline__ void tile_coords(int tile, int MB, int NT, int band_rows, int& mb, int& nt) {
+  const int per_band = band_rows * NT;
+  const int band = tile / per_band, within = tile - band * per_band;
+  const int rows = min(band_rows, MB - band * band_rows);
+  nt = within / rows;
+  mb = band * band_rows + (within - nt * rows);
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&h);
+}
+
+// ---------------------------------------------------------------- epilogues
+// Each epilogue thread owns one accumulator row (TMEM lane) of the 128x256 tile.
+template <int EPI>
+__device__ __forceinline__ void epilogue_tile(const TcArgs& p, uint32_t tmem_acc, int quad, int lane, int mb, int nt) {
+  const int r = quad * 32 + lane;           // row within the tile
+  const int n0 = nt * BN;
+  const uint32_t taddr = tmem_acc + ((uint32_t)(quad * 32) << 16);
+  uint32_t v[32];
+
+  if constexpr (EPI == TC_EPI_LSE) {
+    const int blk = p.blk_off + mb;
+    const bool valid = r < p.blk_n[blk];
+    const long grow = (long)p.blk_row[blk] + r;
+    const int id = valid ? p.ids[grow] : -1;
+    float m2 = -INFINITY, l = 0.f, tg = 0.f;
+    bool has = false;
+    for (int c0 = 0; c0 < BN; c0 += 32) {
+      const int ncl = p.N - (n0 + c0);
+      if (ncl <= 0) break;
+      tc_ld32(taddr + c0, v);
+      tc_wait_ld();
+      float t[32];
+#pragma unroll
+      for (int j = 0; j < 32; ++j) t[j] = __uint_as_float(v[j]) * LOG2E;
+      if (ncl < 32) {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) if (j >= ncl) t[j] = -INFINITY;
+      }
+      float gm = t[0];
+#pragma unroll
+      for (int j = 1; j < 32; ++j) gm = fmaxf(gm, t[j]);
+      const float mnew = fmaxf(m2, gm);
+      float s = 0.f;
+#pragma unroll
+      for (int j = 0; j < 32; ++j) s += ex2(t[j] - mnew);
+      l = l * ex2(m2 - mnew) + s;
+      m2 = mnew;
+      const int lc = id - (n0 + c0);
+      if (lc >= 0 && lc < 32 && lc < ncl) {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) if (j == lc) tg = __uint_as_float(v[j]);
+        has = true;
+      }
+    }
+    const size_t prow = (size_t)blk * BM + r;
+    p.partials[(size_t)nt * p.rows_cap + prow] = make_float2(m2 * LN2, l);
+    if (has) p.tgt[prow] = tg;
+  } else if constexpr (EPI == TC_EPI_DS) {
+    const int blk = p.blk_off + mb;
+    const bool valid = r < p.blk_n[blk];
+    const long grow = (long)p.blk_row[blk] + r;
+    const int id = valid ? p.ids[grow] : -1;
+    const float gg = valid ? p.g[grow] : 0.f;
+    const float L2 = valid ? p.lse[grow] * LOG2E : 0.f;
+    const size_t srow = (size_t)mb * BM + r;
+    __nv_bfloat16* ds_row = p.dS + srow * p.ds_ld;
+    for (int c0 = 0; c0 < BN; c0 += 32) {
+      const int ncl = p.N - (n0 + c0);
+      if (ncl <= 0) break;
+      tc_ld32(taddr + c0, v);
+      tc_wait_ld();
+      float d[32];
+      const int lc = id - (n0 + c0);
+#pragma unroll
+      for (int j = 0; j < 32; ++j) {
+        const float pr = ex2(fmaf(__uint_as_float(v[j]), LOG2E, -L2));
+        const float dj = gg * ((j == lc ? 1.f : 0.f) - pr);
+        d[j] = (valid && gg != 0.f) ? dj : 0.f;
+      }
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        if (q * 8 < ncl) {
+          uint4 w;
+          w.x = pack_bf16x2(d[q * 8 + 0], d[q * 8 + 1]);
+          w.y = pack_bf16x2(d[q * 8 + 2], d[q * 8 + 3]);
+          w.z = pack_bf16x2(d[q * 8 + 4], d[q * 8 + 5]);
+          w.w = pack_bf16x2(d[q * 8 + 6], d[q * 8 + 7]);
+          *reinterpret_cast<uint4*>(ds_row + n0 + c0 + q * 8) = w;
+        }
+      }
+      __nv_bfloat16* dst_col = p.dSt + (size_t)(n0 + c0) * p.dst_ld + srow;
+#pragma unroll
+      for (int j = 0; j < 32; ++j)
+        if (j < ncl) dst_col[(size_t)j * p.dst_ld] = __float2bfloat16_rn(d[j]);
+    }
+  } else if constexpr (EPI == TC_EPI_DH) {
+    const int blk = p.blk_off + mb;
+    const bool valid = r < p.blk_n[blk];
+    const long grow = (long)p.blk_row[blk] + r;
+    __nv_bfloat16* out = p.dHidden + (size_t)grow * p.dh_ld;
+    for (int c0 = 0; c0 < BN; c0 += 32) {
+      const int ncl = p.N - (n0 + c0);
+      if (ncl <= 0) break;
+      tc_ld32(taddr + c0, v);
+      tc_wait_ld();
+      if (valid) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          if (q * 8 < ncl) {
+            uint4 w;
+            w.x = pack_bf16x2(__uint_as_float(v[q * 8 + 0]), __uint_as_float(v[q * 8 + 1]));
+            w.y = pack_bf16x2(__uint_as_float(v[q * 8 + 2]), __uint_as_float(v[q * 8 + 3]));
+            w.z = pack_bf16x2(__uint_as_float(v[q * 8 + 4]), __uint_as_float(v[q * 8 + 5]));
+            w.w = pack_bf16x2(__uint_as_float(v[q * 8 + 6]), __uint_as_float(v[q * 8 + 7]));
+            *reinterpret_cast<uint4*>(out + n0 + c0 + q * 8) = w;
+          }
+        }
+      }
+    }
+  } else {  // TC_EPI_DW
+    const long vrow = (long)mb * BM + r;
+    const bool valid = vrow < p.V;
+    float* out = p.dW + (size_t)vrow * p.dw_ld;
+    for (int c0 = 0; c0 < BN; c0 += 32) {
+      const int ncl = p.N - (n0 + c0);
+      if (ncl <= 0) break;
+      tc_ld32(taddr + c0, v);
+      tc_wait_ld();
+      if (valid) {
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+          if (q * 4 < ncl) {
+            float4* ptr = reinterpret_cast<float4*>(out + n0 + c0 + q * 4);
+            float4 o = *ptr;
+            o.x += __uint_as_float(v[q * 4 + 0]);
+            o.y += __uint_as_float(v[q * 4 + 1]);
+            o.z += __uint_as_float(v[q * 4 + 2]);
+            o.w += __uint_as_float(v[q * 4 + 3]);
+            *ptr = o;
+          }
+        }
+      }
+    }
+  }
+}
+
+// ---------------------------------------------------------------- the kernel
+template <int EPI>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcArgs p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t bar_base = smem_base + STAGES * STAGE_BYTES;
+  // barrier layout (8 B each): full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2]; then tmem slot, abort flag
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+  auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
+  auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
+  uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen_base + STAGES * STAGE_BYTES + 8 * (2 * STAGES + 4));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen_base + STAGES * STAGE_BYTES + 8 * (2 * STAGES + 4) + 8);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  // ---- problem extents (identical in every thread)
+  int live = p.blk_cap;
+  if (p.nblk) live = max(0, min(p.nblk[0] - p.blk_off, p.blk_cap));
+  const int MB = (EPI == TC_EPI_DW) ? p.m_blocks_fixed : live;
+  const int K = (EPI == TC_EPI_DW) ? live * BM : p.K;
+  const int NT = (p.N + BN - 1) / BN;
+  const int nkb = (K + BK - 1) / BK;
+  const int total = (nkb > 0) ? MB * NT : 0;
+  if (total == 0 || (int)blockIdx.x >= total) return;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 128); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    __syncwarp();
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void*)tmem_slot)),
+                 "r"(TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int stage = 0; uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x) {
+        int mb, nt;
+        tile_coords(tile, MB, NT, p.raster_band, mb, nt);
+        const int a_row = (EPI == TC_EPI_LSE || EPI == TC_EPI_DS) ? p.blk_row[p.blk_off + mb] : mb * BM;
+        const int b_row = nt * BN;
+        for (int kb = 0; kb < nkb; ++kb) {
+          if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status))) break;
+          mbar_expect_tx(full_bar(stage), STAGE_BYTES);
+          const uint32_t sa = smem_base + stage * STAGE_BYTES;
+          tma_load_2d(sa, &tmA, kb * BK, a_row, full_bar(stage));
+          tma_load_2d(sa + A_BYTES, &tmB, kb * BK, b_row, full_bar(stage));
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) {   // give copies already in flight time to land before shared memory is released
+        for (int i = 0; i < 200; ++i) __nanosleep(1000);
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc_bf16(BM, BN);
+      int stage = 0; uint32_t phase = 0;
+      int acc = 0; uint32_t acc_phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x) {
+        if (!(ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, p.status))) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+        for (int kb = 0; kb < nkb; ++kb) {
+          if (!(ok = mbar_wait(full_bar(stage), phase, abort_flag, p.status))) break;
+          tc_fence_after();
+          const uint32_t sa = smem_base + stage * STAGE_BYTES;
+          const uint64_t da = make_kmajor_sw128_desc(sa);
+          const uint64_t db = make_kmajor_sw128_desc(sa + A_BYTES);
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k) {
+            // advance 32 B (16 bf16) along K inside the 128 B swizzle row: +2 in the >>4 address field
+            tc_mma_bf16(d_tmem, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (uint32_t)((kb | k) != 0));
+          }
+          tc_commit(empty_bar(stage));
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        tc_commit(tfull_bar(acc));
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      }
+    }
+    __syncwarp();
+  } else {
+    // ------------------------------------------------------------ epilogue warps 2..5
+    const int quad = warp & 3;
+    int acc = 0; uint32_t acc_phase = 0;
+    for (int tile = blockIdx.x; tile < total; tile += gridDim.x) {
+      int mb, nt;
+      tile_coords(tile, MB, NT, p.raster_band, mb, nt);
+      bool ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.status);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      epilogue_tile<EPI>(p, tmem_base + (uint32_t)(acc * BN), quad, lane, mb, nt);
+      tc_fence_before();
+      mbar_arrive(tempty_bar(acc));
+      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+// ---------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = (EncodeTiledFn)ptr;
+  }
+  return fn;
+}
+
+// 2-D bf16 tensor [rows, K] with row pitch `ld` elements; box = [box_rows, 64] elements, 128 B swizzle.
+bool make_tmap(CUtensorMap* tm, const void* base, long rows, long K, long ld, int box_rows) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+  cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+template <int EPI>
+cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, const TcArgs& a, int grid, cudaStream_t s) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  tc_gemm_kernel<EPI><<<grid, NUM_THREADS, SMEM_BYTES, s>>>(tmA, tmB, a);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+int tc_num_sms() {
+  static int n = 0;
+  if (!n) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+  }
+  return n;
+}
+
+cudaError_t launch_tc_gemm(const TcGemm& g, cudaStream_t s) {
+  CUtensorMap tmA, tmB;
+  if (!make_tmap(&tmA, g.A, g.a_rows, g.K, g.a_ld, BM)) return cudaErrorInvalidValue;
+  if (!make_tmap(&tmB, g.B, g.b_rows, g.K, g.b_ld, BN)) return cudaErrorInvalidValue;
+  TcArgs a;
+  a.N = g.N; a.K = g.K; a.m_blocks_fixed = g.m_blocks; a.blk_off = g.blk_off; a.blk_cap = g.blk_cap;
+  a.raster_band = g.raster_band > 0 ? g.raster_band : 16; a.rows_cap = g.rows_cap; a.V = g.V;
+  a.nblk = g.rb.nblk; a.blk_row = g.rb.blk_row; a.blk_n = g.rb.blk_n;
+  a.ids = g.ids; a.lse = g.lse; a.g = g.g; a.partials = g.partials; a.tgt = g.tgt;
+  a.dS = g.dS; a.ds_ld = g.ds_ld; a.dSt = g.dSt; a.dst_ld = g.dst_ld;
+  a.dHidden = g.dHidden; a.dh_ld = g.dh_ld; a.dW = g.dW; a.dw_ld = g.dw_ld; a.status = g.status;
+  const int NT = cdiv(g.N, BN);
+  const long max_tiles = (long)(g.epi == TC_EPI_DW ? g.m_blocks : g.blk_cap) * NT;
+  const int grid = (int)(max_tiles < (long)tc_num_sms() ? (max_tiles > 0 ? max_tiles : 1) : tc_num_sms());
+  switch (g.epi) {
+    case TC_EPI_LSE: return launch_one<TC_EPI_LSE>(tmA, tmB, a, grid, s);
+    case TC_EPI_DS: return launch_one<TC_EPI_DS>(tmA, tmB, a, grid, s);
+    case TC_EPI_DH: return launch_one<TC_EPI_DH>(tmA, tmB, a, grid, s);
+    case TC_EPI_DW: return launch_one<TC_EPI_DW>(tmA, tmB, a, grid, s);
+  }
+  return cudaErrorInvalidValue;
+}
+
+}  // namespace trl

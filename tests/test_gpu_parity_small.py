@@ -1,0 +1,189 @@
+"""CUDA path vs fp64 oracle, element by element, on shapes the oracle finishes in seconds.
+All calls go through the C ABI (ctypes binding)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import trl_oracle as orc
+from paper_2510_17891_b200 import synth
+from tests._util import f64, oracle_inputs, rel_fro, TOL_LOGP, TOL_LOSS, TOL_GRAD
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def trl():
+    import paper_2510_17891_b200 as t
+    t.load_library()
+    assert torch.cuda.is_available()
+    return t
+
+
+def run_and_compare(trl, w, batch=None, explicit_old=False, alpha=0.1, eps=0.2, adv_mode=0):
+    dev = "cuda:0"
+    batch = synth.make_batch(w, device=dev) if batch is None else batch
+    oi = oracle_inputs(batch)
+    old_logp_o = None
+    old_logp_g = None
+    if explicit_old:      # old logp = oracle logp + N(0, sigma): an input to both sides
+        lp, _ = orc.token_logprobs(oi["hidden"], oi["W"], oi["ids"], oi["lens"], w.T)
+        old_logp_o = (lp + oi["old_noise"]).astype(np.float32).astype(np.float64)
+        old_logp_g = torch.tensor(old_logp_o, dtype=torch.float32, device=dev)
+    ref = orc.full_step(oi["hidden"], oi["W"], oi["hidden_old"], oi["W_old"], oi["ids"], oi["lens"], oi["bnd"],
+                        oi["r_plan"], oi["r_code"], w.P, w.G, w.T, eps, eps, alpha, adv_mode, old_logp=old_logp_o)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    out = trl.hrd_pg_step(batch, w.P, w.G, w.T, eps, eps, alpha, adv_mode, old_logp=old_logp_g, status=status)
+    torch.cuda.synchronize()
+    trl.check_status(status)
+    hrd = out["hrd"]
+    # integers: bit exact
+    np.testing.assert_array_equal(hrd["seg"].cpu().numpy(), ref["seg"])
+    np.testing.assert_array_equal(hrd["n_plan"].cpu().numpy(), ref["n_plan"])
+    np.testing.assert_array_equal(hrd["n_code"].cpu().numpy(), ref["n_code"])
+    assert int(hrd["n_valid"].item()) == ref["n_valid"]
+    np.testing.assert_allclose(f64(hrd["A_plan"]), ref["A_plan"], rtol=1e-6, atol=1e-7)
+    np.testing.assert_allclose(f64(hrd["A_code"]), ref["A_code"], rtol=1e-6, atol=1e-7)
+    np.testing.assert_allclose(f64(hrd["adv"]), ref["adv"], rtol=1e-6, atol=1e-7)
+    # floating point
+    assert np.abs(f64(out["logp"]) - ref["logp"]).max() <= TOL_LOGP
+    assert np.abs(f64(out["lse"]) - ref["lse"]).max() <= TOL_LOGP
+    if not explicit_old:
+        assert np.abs(f64(out["old_logp"]) - ref["old_logp"]).max() <= TOL_LOGP
+    assert abs(float(out["loss"]) - ref["loss"]) <= TOL_LOSS * abs(ref["loss"]) + 1e-9
+    valid = ref["seg"] != 0
+    assert not f64(out["g"])[~valid].any() and not f64(out["logp"])[~valid].any()
+    assert rel_fro(f64(out["g"]), ref["g"]) <= TOL_GRAD
+    dH = f64(out["dHidden"])
+    assert not dH[~valid].any()
+    if np.linalg.norm(ref["dHidden"]) > 0:
+        assert rel_fro(dH, ref["dHidden"]) <= TOL_GRAD
+        assert rel_fro(f64(out["dW"]), ref["dW"]) <= TOL_GRAD
+    else:
+        assert not dH.any() and not f64(out["dW"]).any()
+    st = f64(out["stats"])
+    np.testing.assert_allclose(st[:3], ref["stats"][:3], atol=2e-3)
+    assert st[3] == ref["stats"][3]
+    return out, ref
+
+
+def test_config0_f32_end_to_end(trl):
+    run_and_compare(trl, synth.CONFIGS[0])
+    run_and_compare(trl, synth.CONFIGS[0], explicit_old=True)
+
+
+def test_config0_literal_boundary_reading(trl):
+    run_and_compare(trl, synth.scaled(synth.CONFIGS[0], name="cfg0_bnd_of_T", bnd_of_T=True), explicit_old=True)
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_ragged_multi_tile(trl, dtype):
+    # rows: 3 blocks per rollout with a ragged tail; K: 5 k-blocks; V: 4 tiles, the last one partial
+    w = synth.scaled(synth.CONFIGS[2], name=f"twin_ragged_{dtype}", P=2, G=4, T=300, H=320, V=1000, dtype=dtype)
+    run_and_compare(trl, w)
+    run_and_compare(trl, w, explicit_old=True, alpha=0.5, eps=0.1)
+
+
+def test_bf16_many_tiles_real_plan_reward(trl):
+    # more tiles than SMs in the forward, several waves, 2 raster bands; non-binary plan reward
+    w = synth.scaled(synth.CONFIGS[2], name="twin_wide", P=3, G=6, T=384, H=512, V=3000, real_plan_reward=True,
+                     len_lo=0.1)
+    run_and_compare(trl, w)
+
+
+def test_long_reasoning_twin_bf16(trl):
+    w = synth.scaled(synth.CONFIGS[3], name="twin_cfg3", P=2, G=8, T=512, H=256, V=2048)
+    run_and_compare(trl, w)
+    run_and_compare(trl, synth.scaled(w, name="twin_cfg3_lit", bnd_of_T=True))
+
+
+def test_sweep_twin_degenerate_groups_and_std_mode(trl):
+    for G in (4, 16):
+        w = synth.scaled(synth.CONFIGS[2], name=f"twin_sweep_G{G}", P=64 // G, G=G, T=128, H=256, V=1536,
+                         degenerate_frac=0.25)
+        run_and_compare(trl, w)
+    run_and_compare(trl, synth.scaled(synth.CONFIGS[2], name="twin_std", P=4, G=4, T=128, H=256, V=1024), adv_mode=1)
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_edge_cases_empty_rollouts_and_boundaries(trl, dtype):
+    w = synth.scaled(synth.CONFIGS[2], name=f"edge_{dtype}", P=2, G=4, T=160, H=128, V=512, dtype=dtype)
+    batch = synth.make_batch(w, device="cuda:0")
+    lens = torch.tensor([0, 160, 1, 128, 129, 77, 0, 5], dtype=torch.int32)
+    bnd = torch.tensor([0, 0, 1, 128, 64, 77, 0, 2], dtype=torch.int32)   # no plan / no code / both
+    batch["lens"], batch["bnd"] = lens.cuda(), bnd.cuda()
+    run_and_compare(trl, w, batch=batch)
+    # everything padded: all outputs zero
+    batch["lens"], batch["bnd"] = torch.zeros(8, dtype=torch.int32).cuda(), torch.zeros(8, dtype=torch.int32).cuda()
+    out, _ = run_and_compare(trl, w, batch=batch)
+    assert float(out["loss"]) == 0.0
+
+
+def test_all_equal_rewards_give_exact_zero(trl):
+    w = synth.scaled(synth.CONFIGS[2], name="degenerate_all", P=2, G=4, T=128, H=128, V=512)
+    batch = synth.make_batch(w, device="cuda:0")
+    batch["r_plan"] = torch.tensor([0.7] * 4 + [1.3] * 4, device="cuda:0")
+    batch["r_code"] = torch.tensor([1.0] * 4 + [0.0] * 4, device="cuda:0")
+    out, _ = run_and_compare(trl, w, batch=batch)
+    assert float(out["loss"]) == 0.0 and not out["g"].any() and not out["dW"].any() and not out["dHidden"].any()
+
+
+def test_group_size_one(trl):
+    w = synth.scaled(synth.CONFIGS[0], name="g1", P=6, G=1, T=64, H=64, V=256)
+    out, _ = run_and_compare(trl, w)
+    assert float(out["loss"]) == 0.0
+
+
+def test_uniform_logits_closed_form(trl):
+    # W = 0: logp = -ln V exactly representable to fp32 rounding on both paths
+    for dtype, tdt in (("bf16", torch.bfloat16), ("f32", torch.float32)):
+        w = synth.scaled(synth.CONFIGS[2], name="uniform", P=1, G=2, T=128, H=64, V=1000, dtype=dtype)
+        batch = synth.make_batch(w, device="cuda:0")
+        batch["W"] = torch.zeros_like(batch["W"])
+        logp, lse = trl.trl_token_logprobs(batch["hidden"], batch["W"], batch["ids"], batch["lens"], w.T)
+        torch.cuda.synchronize()
+        L = int(batch["lens"][0])
+        assert abs(float(lse[0]) - np.log(1000.0)) < 1e-5 and abs(float(logp[L - 1]) + np.log(1000.0)) < 1e-5
+
+
+def test_device_detected_bad_inputs_set_status_without_faulting(trl):
+    w = synth.scaled(synth.CONFIGS[2], name="bad", P=1, G=2, T=128, H=64, V=512)
+    batch = synth.make_batch(w, device="cuda:0")
+    batch["ids"][3] = 100000          # outside [0, V)
+    batch["lens"][:] = torch.tensor([128, 90], dtype=torch.int32)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda:0")
+    logp, _ = trl.trl_token_logprobs(batch["hidden"], batch["W"], batch["ids"], batch["lens"], w.T, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) & (1 << 7) and float(logp[3]) == 0.0
+    with pytest.raises(trl.TrlError):
+        trl.check_status(status)
+    status.zero_()
+    batch["bnd"][0] = 500             # beyond len
+    trl.trl_hrd_advantages(batch["r_plan"], batch["r_code"], batch["lens"], batch["bnd"], 1, 2, w.T, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) & (1 << 7)
+
+
+def test_host_argument_errors(trl):
+    w = synth.scaled(synth.CONFIGS[2], name="args", P=1, G=2, T=128, H=64, V=512)
+    batch = synth.make_batch(w, device="cuda:0")
+    tiny = torch.empty(256, dtype=torch.uint8, device="cuda:0")
+    with pytest.raises(trl.TrlError, match="workspace"):
+        trl.trl_token_logprobs(batch["hidden"], batch["W"], batch["ids"], batch["lens"], w.T, workspace=tiny)
+    with pytest.raises(trl.TrlError, match="shape"):
+        trl.trl_token_logprobs(batch["hidden"][:, :60].contiguous(), batch["W"][:, :60].contiguous(), batch["ids"],
+                               batch["lens"], w.T)      # H % 8 != 0 in bf16
+
+
+def test_minimum_workspace_gives_same_backward(trl):
+    # chunked backward (one 128-row block per chunk) equals the one-chunk result
+    w = synth.scaled(synth.CONFIGS[2], name="chunks", P=1, G=3, T=200, H=128, V=512)
+    batch = synth.make_batch(w, device="cuda:0")
+    logp, lse = trl.trl_token_logprobs(batch["hidden"], batch["W"], batch["ids"], batch["lens"], w.T)
+    g = torch.randn(w.N, device="cuda:0") * (torch.arange(w.N, device="cuda:0") % w.T < batch["lens"].repeat_interleave(w.T))
+    dH1, dW1 = trl.trl_pg_loss_bwd(batch["hidden"], batch["W"], batch["ids"], batch["lens"], lse, g, w.T)
+    nmin = trl.trl_workspace_bytes_min(trl.TRL_CALL_PG_LOSS_BWD, w.B, w.T, w.H, w.V, trl.TRL_BF16)
+    ws = torch.empty(nmin, dtype=torch.uint8, device="cuda:0")
+    dH2, dW2 = trl.trl_pg_loss_bwd(batch["hidden"], batch["W"], batch["ids"], batch["lens"], lse, g, w.T, workspace=ws)
+    torch.cuda.synchronize()
+    assert torch.equal(dH1, dH2)
+    assert rel_fro(f64(dW2), f64(dW1)) < 1e-5
