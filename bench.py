@@ -1,0 +1,326 @@
+#!/usr/bin/env python
+"""Benchmark of the HRD policy-gradient scoring path on B200.
+
+A step is one pass of the whole path over one synthetic batch: scoring under the current
+and the old policy, HRD advantages, clipped surrogate, backward to dHidden and dW.
+Metric: scored (valid) rollout tokens per second, fwd+bwd, at H=4096, V=151,936.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+N > 1 is launched with torch.distributed.run (one rank per GPU); ranks process independent
+batches (weak scaling, no data-path collective); time is the max over ranks.
+`--impl reference` times the fp64 CPU oracle on a bounded sample of the same workload.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "scored_rollout_tokens_per_sec_fwd_bwd"
+UNIT = "tokens/s"
+WORKLOAD_ID = 2          # 8B-scale fwd+bwd: 8 prompts x 8 rollouts, T=2048, H=4096, V=151,936
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm_gbs=p["hbm_gbs"], bf16_burst=p["bf16_tflops"], bf16_sustained=p["bf16_tflops_sustained"],
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16_burst=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu_index = gpu_index
+        self.lines = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.gpu_index), "-lms", "200"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, power, reasons = [], None, [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); smax = float(f[2]); power.append(float(f[3]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return dict(sm_mhz=statistics.median(sm) if sm else None, sm_max_mhz=smax,
+                    power_w_max=max(power) if power else None, samples=len(sm), reasons=sorted(reasons))
+
+
+def oracle_sample_throughput(w, rollouts, T_sample, seed_offset=0):
+    """Time the fp64 oracle, as it stands, on `rollouts` rollouts of length T_sample with the
+    full H and V of workload `w`.  Returns (tokens/s, tokens, seconds, threads)."""
+    import numpy as np
+    import torch
+    from threadpoolctl import threadpool_info
+    from oracle import trl_oracle as orc
+    from paper_2510_17891_b200 import synth
+    ws = synth.scaled(w, name=w.name + "_cpu_sample", P=1, G=rollouts, T=T_sample)
+    b = synth.make_batch(ws, device="cpu", seed_offset=seed_offset)
+    f64 = lambda t: t.to(torch.float64).numpy()
+    hidden, W, W_old = f64(b["hidden"]), f64(b["W"]), f64(b["W_old"])
+    ids, lens, bnd = b["ids"].numpy(), b["lens"].numpy(), b["bnd"].numpy()
+    rp, rc = f64(b["r_plan"]), f64(b["r_code"])
+    t0 = time.perf_counter()
+    orc.full_step(hidden, W, hidden, W_old, ids, lens, bnd, rp, rc, 1, rollouts, T_sample)
+    dt = time.perf_counter() - t0
+    threads = max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
+    tokens = int(lens.sum())
+    return tokens / dt, tokens, dt, threads
+
+
+def run_reference(args, rank, world):
+    """Reference arm = the oracle on the host cores (rank 0 only)."""
+    if rank != 0:
+        return
+    from paper_2510_17891_b200 import synth
+    w = synth.CONFIGS[WORKLOAD_ID]
+    rollouts, T_sample = 2, 16
+    for i in range(args.warmup):
+        oracle_sample_throughput(w, 1, 4, seed_offset=100 + i)
+    tok = sec = 0
+    threads = 1
+    for i in range(args.steps):
+        _, t, s, threads = oracle_sample_throughput(w, rollouts, T_sample, seed_offset=i)
+        tok += t; sec += s
+    value = tok / sec
+    sample = (f"{rollouts} rollouts x T={T_sample} per step (valid tokens only), full H={w.H} V={w.V}, "
+              f"policy + old-policy scoring, advantages, loss, backward in numpy fp64")
+    line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps, warmup=args.warmup,
+                ms_per_step=1e3 * sec / max(args.steps, 1), higher_is_better=True, scaling="weak", vs_baseline=None,
+                dtype="f64", data="synthetic", impl="reference",
+                config=dict(workload=w.name, P=w.P, G=w.G, T=w.T, H=w.H, V=w.V, note="oracle on a bounded sample"),
+                cpu_baseline=dict(value=value, unit=UNIT, cores=threads, kind="oracle", sample=sample),
+                e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0),
+                gpu_launches=0)
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=8)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", type=int, default=WORKLOAD_ID, help="config number (default: the metric's)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+        return
+
+    import torch
+    import paper_2510_17891_b200 as trl
+    from paper_2510_17891_b200 import synth
+    trl.load_library()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    w = synth.CONFIGS[args.workload]
+    peaks = load_peaks()
+    batch = synth.make_batch(w, device=dev, seed_offset=rank)
+    batch["hidden_old"] = batch["hidden"].clone()        # the old policy's own activation buffer
+    B, T, H, V, P, G = w.B, w.T, w.H, w.V, w.P, w.G
+    n_valid = int(batch["lens"].sum().item())
+    dt_code = trl.TRL_BF16 if w.dtype == "bf16" else trl.TRL_F32
+
+    # preallocated outputs and workspaces (the library allocates nothing)
+    f32 = dict(dtype=torch.float32, device=dev)
+    ws = lambda call: torch.empty(max(trl.trl_workspace_bytes(call, B, T, H, V, dt_code), 256), dtype=torch.uint8, device=dev)
+    bufs = dict(logp=torch.empty(B * T, **f32), lse=torch.empty(B * T, **f32), old_logp=torch.empty(B * T, **f32),
+                old_lse=torch.empty(B * T, **f32), loss=torch.empty(1, **f32), g=torch.empty(B * T, **f32),
+                stats=torch.empty(4, **f32), dHidden=torch.empty_like(batch["hidden"]),
+                dW=torch.empty(V, H, **f32), ws_fwd=ws(trl.TRL_CALL_TOKEN_LOGPROBS),
+                ws_loss=ws(trl.TRL_CALL_PG_LOSS_FWD), ws_bwd=ws(trl.TRL_CALL_PG_LOSS_BWD))
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step(ev=None):
+        """The five C-ABI calls of one pass.  `ev` collects CUDA events around each call."""
+        mark = (lambda: None) if ev is None else (lambda: ev.append(_rec()))
+        mark()
+        trl.trl_token_logprobs(batch["hidden"], batch["W"], batch["ids"], batch["lens"], T, bufs["logp"], bufs["lse"],
+                               bufs["ws_fwd"], status, stream)
+        mark()
+        trl.trl_token_logprobs(batch["hidden_old"], batch["W_old"], batch["ids"], batch["lens"], T, bufs["old_logp"],
+                               bufs["old_lse"], bufs["ws_fwd"], status, stream)
+        mark()
+        hrd = trl.trl_hrd_advantages(batch["r_plan"], batch["r_code"], batch["lens"], batch["bnd"], P, G, T, 0,
+                                     bufs.get("hrd"), status, stream)
+        bufs["hrd"] = hrd
+        mark()
+        trl.trl_pg_loss_fwd(bufs["logp"], bufs["old_logp"], hrd["adv"], hrd["seg"], batch["lens"], P, G, T, 0.2, 0.2, 0.1,
+                            bufs["loss"], bufs["g"], bufs["stats"], bufs["ws_loss"], status, stream)
+        mark()
+        trl.trl_pg_loss_bwd(batch["hidden"], batch["W"], batch["ids"], batch["lens"], bufs["lse"], bufs["g"], T,
+                            bufs["dHidden"], bufs["dW"], bufs["ws_bwd"], status, stream)
+        mark()
+
+    def _rec():
+        e = torch.cuda.Event(enable_timing=True)
+        e.record(stream)
+        return e
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    trl.check_status(status)
+
+    launches0 = trl.trl_kernel_launches()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    barrier()
+    call_events = []
+    t_start = _rec()
+    for _ in range(args.steps):
+        ev = []
+        step(ev)
+        call_events.append(ev)
+    t_end = _rec()
+    barrier()
+    clocks = sampler.stop()
+    launches = trl.trl_kernel_launches() - launches0
+    trl.check_status(status)
+    elapsed_ms = t_start.elapsed_time(t_end)
+    if dist is not None:
+        t = torch.tensor([elapsed_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(t.item())
+        tot = torch.tensor([n_valid], device=dev, dtype=torch.int64)
+        dist.all_reduce(tot)
+        total_valid = int(tot.item())
+    else:
+        total_valid = n_valid
+    value = total_valid * args.steps / (elapsed_ms * 1e-3)
+
+    # per-call device times (this rank), averaged over the timed steps
+    names = ["token_logprobs_policy", "token_logprobs_old", "hrd_advantages", "pg_loss_fwd", "pg_loss_bwd"]
+    call_ms = {n: statistics.mean(ev[i].elapsed_time(ev[i + 1]) for ev in call_events) for i, n in enumerate(names)}
+
+    # ---- end-to-end: host buffers in, loss out, copies inside the timed region
+    host = {k: batch[k].cpu().pin_memory() for k in ("hidden", "hidden_old", "ids", "lens", "bnd", "r_plan", "r_code")}
+    host_out = torch.empty(5, dtype=torch.float32).pin_memory()
+    h2d = sum(v.numel() * v.element_size() for v in host.values())
+    d2h = host_out.numel() * 4
+    e2e_steps = max(2, min(args.steps, 4))
+
+    def e2e_step():
+        for k, v in host.items():
+            batch[k].copy_(v, non_blocking=True)
+        step()
+        host_out[:1].copy_(bufs["loss"], non_blocking=True)
+        host_out[1:].copy_(bufs["stats"], non_blocking=True)
+        torch.cuda.synchronize()
+
+    e2e_step()
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        e2e_step()
+    e2e_s = time.perf_counter() - t0
+    if dist is not None:
+        t = torch.tensor([e2e_s], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    e2e_value = total_valid * e2e_steps / e2e_s
+
+    # ---- roofline of the dominant kernel: the tcgen05 GEMM with the log-sum-exp epilogue
+    # (2 launches per step, 40 % of the executed FLOPs).  Its launch is timed through the
+    # trl_token_logprobs call that contains it (plus two sub-millisecond helper kernels).
+    flops_fwd = 2.0 * H * V * n_valid
+    t_fwd_ms = 0.5 * (call_ms["token_logprobs_policy"] + call_ms["token_logprobs_old"])
+    achieved = flops_fwd / (t_fwd_ms * 1e-3) / 1e12
+    peak = peaks["bf16_sustained"]
+    roofline = dict(bound="tensor", kernel="tc_gemm_kernel<LSE> (inside trl_token_logprobs)", achieved=achieved,
+                    peak=peak, unit="TFLOP/s", frac=achieved / peak, traffic=None,
+                    peak_source=f"{peaks['source']} sustained cuBLAS bf16")
+    bwd_alg = 4.0 * H * V * n_valid / (call_ms["pg_loss_bwd"] * 1e-3) / 1e12
+    step_alg = 6.0 * H * V * value / world / 1e12
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        v_cpu, tok, sec, threads = oracle_sample_throughput(w, 2, 24)
+        cpu_baseline = dict(value=v_cpu, unit=UNIT, cores=threads, kind="oracle",
+                            sample=f"2 rollouts x T=24 ({tok} valid tokens, {sec:.1f} s), full H={H} V={V}, whole path in numpy fp64")
+
+    if rank == 0:
+        line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=max(args.warmup, 3),
+                    ms_per_step=elapsed_ms / args.steps, higher_is_better=True, scaling="weak", vs_baseline=None,
+                    dtype=w.dtype, data="synthetic",
+                    config=dict(workload=w.name, P=P, G=G, T=T, H=H, V=V, valid_tokens_per_rank=n_valid,
+                                padded_rows_per_rank=B * T, l2="inputs larger than L2 (W alone is 1.2 GB); no flush",
+                                parallelism=f"replicas x{world} (independent batches)"),
+                    pct_of_bf16_peak_6NHV=dict(sustained=100 * step_alg / peaks["bf16_sustained"],
+                                               burst=100 * step_alg / peaks["bf16_burst"], nominal=100 * step_alg / 2250.0,
+                                               note="6*H*V FLOP per scored token over the whole step (which also scores the old policy)"),
+                    roofline=roofline,
+                    calls_ms=call_ms,
+                    bwd_algorithmic_tflops=bwd_alg,
+                    e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
+                             steps=e2e_steps),
+                    gpu_launches=int(launches),
+                    clocks=clocks,
+                    cpu_baseline=cpu_baseline,
+                    loss=float(host_out[0]))
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -157,6 +157,11 @@ int trl_pg_loss_bwd(const void* hidden, const void* W, const int32_t* ids, const
                     void* dHidden, float* dW,
                     void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream);
 
+/* Number of kernels this library has enqueued so far in this process (all streams, all
+ * calls; memsets are not counted).  Host-side statistic used by the benchmark; there is no
+ * counterpart in the paper. */
+unsigned long long trl_kernel_launches(void);
+
 /* Host string for a status code (static storage). */
 const char* trl_status_string(int status);
 

@@ -97,6 +97,8 @@ size_t trl_workspace_bytes_min(int which_call, int B, int T, int H, int V, trl_d
   return ws_bytes(which_call, B, T, H, V, dt, true);
 }
 
+unsigned long long trl_kernel_launches(void) { return launches_so_far(); }
+
 const char* trl_status_string(int status) {
   switch (status) {
     case TRL_OK: return "ok";

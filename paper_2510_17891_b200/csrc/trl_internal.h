@@ -11,6 +11,10 @@ namespace trl {
 
 constexpr int kRowBlock = 128;   // rows per row block = TMEM lanes of one accumulator tile
 
+// process-wide count of kernels this library has enqueued (statistics only)
+void note_launch(int n = 1);
+unsigned long long launches_so_far();
+
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline int cdiv(int a, int b) { return (a + b - 1) / b; }
 

@@ -63,6 +63,7 @@ __global__ void __launch_bounds__(256) simt_gemm_kernel(SimtGemm p) {
 void launch_simt_gemm(const SimtGemm& p, cudaStream_t s) {
   dim3 grid(cdiv(p.N, BN), cdiv(p.M, BM));
   simt_gemm_kernel<<<grid, 256, 0, s>>>(p);
+  note_launch();
 }
 
 }  // namespace trl

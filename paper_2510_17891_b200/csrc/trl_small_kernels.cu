@@ -1,9 +1,15 @@
 // Memory-bound kernels of the HRD policy-gradient path: row-block construction, HRD
 // advantages (Section 2.3, Eq. 2), the clipped surrogate and its derivative, the merge of
 // per-vocabulary-tile log-sum-exp partials, and layout helpers.
+#include <atomic>
+
 #include "trl_internal.h"
 
 namespace trl {
+
+static std::atomic<unsigned long long> g_launches{0};
+void note_launch(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
+unsigned long long launches_so_far() { return g_launches.load(std::memory_order_relaxed); }
 
 __device__ __forceinline__ void flag_status(int32_t* status, int code) {
   if (status) atomicOr(status, 1 << code);
@@ -66,6 +72,7 @@ __global__ void build_row_blocks_kernel(const int32_t* __restrict__ len, int B, 
 
 void launch_build_row_blocks(const int32_t* len, int B, int T, RowBlocks rb, int32_t* status, cudaStream_t s) {
   build_row_blocks_kernel<<<1, 1024, 0, s>>>(len, B, T, rb, status);
+  note_launch();
 }
 
 // ------------------------------------------------------------------------------------
@@ -162,6 +169,7 @@ void launch_hrd_advantages(const float* r_plan, const float* r_code, const int32
   dim3 grid(cdiv(T, kAdvTile), P * G);
   hrd_adv_kernel<<<grid, 256, 0, s>>>(r_plan, r_code, len, bnd, P, G, T, adv_mode, A_plan, A_code, seg, adv,
                                       n_plan, n_code, n_valid, status);
+  note_launch();
 }
 
 // ------------------------------------------------------------------------------------
@@ -255,7 +263,9 @@ void launch_pg_loss(const float* logp, const float* old_logp, const float* adv, 
   const int tiles = pg_loss_tiles(T);
   dim3 grid(tiles, P * G);
   pg_loss_stage1_kernel<<<grid, 256, 0, s>>>(logp, old_logp, adv, seg, len, P, G, T, cfg, g, partials);
+  note_launch();
   pg_loss_stage2_kernel<<<1, 256, 0, s>>>(partials, len, P, G, T, tiles, loss, stats);
+  note_launch();
 }
 
 // ------------------------------------------------------------------------------------
@@ -297,6 +307,7 @@ void launch_merge_lse(const float2* partials, const float* tgt, int n_tiles, int
   const size_t N = (size_t)B * T;
   merge_lse_kernel<<<(unsigned)((N + 255) / 256), 256, 0, s>>>(partials, tgt, n_tiles, rows_cap, rb, ids, len, B, T,
                                                                V, logp, lse, status);
+  note_launch();
 }
 
 // ------------------------------------------------------------------------------------
@@ -321,6 +332,7 @@ __global__ void __launch_bounds__(256) transpose_bf16_kernel(const __nv_bfloat16
 void launch_transpose_bf16(const __nv_bfloat16* in, __nv_bfloat16* out, int rows, int cols, cudaStream_t s) {
   dim3 grid(cdiv(cols, 64), cdiv(rows, 64));
   transpose_bf16_kernel<<<grid, 256, 0, s>>>(in, out, rows, cols);
+  note_launch();
 }
 
 // Xt [H, R]: column r is hidden row (block blk_off + r/128, lane r%128) or 0 if not live.
@@ -350,6 +362,7 @@ void launch_gather_transpose_bf16(const __nv_bfloat16* hidden, __nv_bfloat16* Xt
                                   int blk_off, cudaStream_t s) {
   dim3 grid(cdiv(H, 64), cdiv(R, 64));
   gather_transpose_bf16_kernel<<<grid, 256, 0, s>>>(hidden, Xt, H, R, rb, blk_off);
+  note_launch();
 }
 
 // ------------------------------------------------------------------------------------
@@ -370,6 +383,7 @@ __global__ void pack_rows_f32_kernel(const float* __restrict__ hidden, float* __
 }
 void launch_pack_rows_f32(const float* hidden, float* Xp, int H, int R, RowBlocks rb, int blk_off, cudaStream_t s) {
   pack_rows_f32_kernel<<<R, 128, 0, s>>>(hidden, Xp, H, R, rb, blk_off);
+  note_launch();
 }
 
 __device__ __forceinline__ float block_reduce(float v, bool is_max, float* sh) {
@@ -412,6 +426,7 @@ __global__ void __launch_bounds__(256) row_lse_f32_kernel(const float* __restric
 void launch_row_lse_f32(const float* S, int V, int R, RowBlocks rb, int blk_off, const int32_t* ids, float* logp,
                         float* lse, int32_t* status, cudaStream_t s) {
   row_lse_f32_kernel<<<R, 256, 0, s>>>(S, V, R, rb, blk_off, ids, logp, lse, status);
+  note_launch();
 }
 
 __global__ void __launch_bounds__(256) ds_inplace_f32_kernel(float* __restrict__ S, int V, int R, RowBlocks rb,
@@ -432,6 +447,7 @@ __global__ void __launch_bounds__(256) ds_inplace_f32_kernel(float* __restrict__
 void launch_ds_inplace_f32(float* S, int V, int R, RowBlocks rb, int blk_off, const int32_t* ids, const float* lse,
                            const float* g, cudaStream_t s) {
   ds_inplace_f32_kernel<<<R, 256, 0, s>>>(S, V, R, rb, blk_off, ids, lse, g);
+  note_launch();
 }
 
 __global__ void scatter_rows_f32_kernel(const float* __restrict__ dHp, float* __restrict__ dHidden, int H, int R,
@@ -444,6 +460,7 @@ __global__ void scatter_rows_f32_kernel(const float* __restrict__ dHp, float* __
 void launch_scatter_rows_f32(const float* dHp, float* dHidden, int H, int R, RowBlocks rb, int blk_off,
                              cudaStream_t s) {
   scatter_rows_f32_kernel<<<R, 128, 0, s>>>(dHp, dHidden, H, R, rb, blk_off);
+  note_launch();
 }
 
 __global__ void zero_padded_f32_kernel(float* __restrict__ a, float* __restrict__ b, const int32_t* __restrict__ len,
@@ -456,6 +473,7 @@ __global__ void zero_padded_f32_kernel(float* __restrict__ a, float* __restrict_
 void launch_zero_padded_f32(float* a, float* b, const int32_t* len, int B, int T, cudaStream_t s) {
   const size_t N = (size_t)B * T;
   zero_padded_f32_kernel<<<(unsigned)((N + 255) / 256), 256, 0, s>>>(a, b, len, B, T);
+  note_launch();
 }
 
 }  // namespace trl

@@ -455,6 +455,7 @@ cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, const TcA
     attr_set = true;
   }
   tc_gemm_kernel<EPI><<<grid, NUM_THREADS, SMEM_BYTES, s>>>(tmA, tmB, a);
+  note_launch();
   return cudaGetLastError();
 }
 
