@@ -157,6 +157,30 @@ int trl_pg_loss_bwd(const void* hidden, const void* W, const int32_t* ids, const
                     void* dHidden, float* dW,
                     void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream);
 
+/*
+ * Same computation and outputs as trl_pg_loss_fwd, for callers that cannot allocate device
+ * memory and so cannot supply its workspace: a trainer whose memory arena already owns the
+ * whole device (a further cudaMalloc fails or fragments it), or a step loop that cannot
+ * afford the device-wide synchronisation cudaMalloc / cudaFree imply.  (The paper has no
+ * counterpart to this call; it exists for such callers only.)
+ *
+ * The partial sums live in a fixed 1 MiB array inside the library image (every GPU that
+ * loads the library holds it until the process exits).  Limit: P*G*ceil(T/4096) <= 65536,
+ * otherwise TRL_ERR_WORKSPACE_TOO_SMALL is returned and nothing is launched.  The call
+ * performs no cudaMalloc / cudaFree and calls no allocating routine; inputs and outputs are
+ * still the caller's device buffers.
+ *
+ * The first call on each device looks up the array's device address (the device must be
+ * current); make that first call before starting any stream capture.  All calls on a
+ * device share the one array: two calls whose kernels may overlap on the GPU (different
+ * streams without an ordering between them) race on it and give wrong sums; calls on one
+ * stream, or otherwise ordered, are fine.  The array keeps whatever the last call left in
+ * it; every value a call reads it has written itself first, so nothing needs clearing.
+ */
+int trl_pg_loss_fwd_static(const float* logp, const float* old_logp, const float* adv, const uint8_t* seg,
+                           const int32_t* len, int P, int G, int T, trl_pg_config cfg,
+                           float* loss, float* g, float* stats, int32_t* status_dev, void* stream);
+
 /* Number of kernels this library has enqueued so far in this process (all streams, all
  * calls; memsets are not counted).  Host-side statistic used by the benchmark; there is no
  * counterpart in the paper. */

@@ -34,6 +34,7 @@ _SIGNATURES = {
     "trl_token_logprobs": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _vp, _vp, _sz, _vp, _vp]),
     "trl_hrd_advantages": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "trl_pg_loss_fwd": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, PgConfig, _vp, _vp, _vp, _vp, _sz, _vp, _vp]),
+    "trl_pg_loss_fwd_static": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, PgConfig, _vp, _vp, _vp, _vp, _vp]),
     "trl_pg_loss_bwd": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _vp, _vp, _sz, _vp, _vp]),
 }
 
@@ -170,6 +171,20 @@ def trl_pg_loss_fwd(logp, old_logp, adv, seg, lens, P, G, T, eps_lo=0.2, eps_hi=
                                         PgConfig(eps_lo, eps_hi, alpha), _ptr(loss), _ptr(g), _ptr(stats),
                                         _ptr(workspace), workspace.numel(), _ptr(status), _stream(stream))
     _check(rc, "trl_pg_loss_fwd")
+    return loss, g, stats
+
+
+def trl_pg_loss_fwd_static(logp, old_logp, adv, seg, lens, P, G, T, loss, g, stats, eps_lo=0.2, eps_hi=0.2,
+                           alpha=0.1, status=None, stream=None):
+    """trl_pg_loss_fwd for callers that cannot allocate: the scratch is a fixed array inside the
+    library, and this wrapper allocates nothing either, so `loss` [1], `g` [P*G*T] and `stats`
+    [4] (or None) must be passed in.  Limit P*G*ceil(T/4096) <= 65536.  Calls that may overlap
+    on the GPU must not share a device.  Returns (loss, g, stats)."""
+    _dev(logp, old_logp, adv, seg, lens, loss, g, stats, status)
+    rc = load_library().trl_pg_loss_fwd_static(_ptr(logp), _ptr(old_logp), _ptr(adv), _ptr(seg), _ptr(lens), P, G, T,
+                                               PgConfig(eps_lo, eps_hi, alpha), _ptr(loss), _ptr(g), _ptr(stats),
+                                               _ptr(status), _stream(stream))
+    _check(rc, "trl_pg_loss_fwd_static")
     return loss, g, stats
 
 
