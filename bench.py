@@ -155,7 +155,7 @@ def main():
 
     import torch
     import paper_2510_17891_b200 as trl
-    from paper_2510_17891_b200 import synth
+    from paper_2510_17891_b200 import synth, dp
     trl.load_library()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
@@ -168,7 +168,7 @@ def main():
 
     w = synth.CONFIGS[args.workload]
     peaks = load_peaks()
-    batch = synth.make_batch(w, device=dev, seed_offset=rank)
+    batch = synth.make_batch(w, device=dev, seed_offset=dp.rank_seed_offset(rank))
     batch["hidden_old"] = batch["hidden"].clone()        # the old policy's own activation buffer
     B, T, H, V, P, G = w.B, w.T, w.H, w.V, w.P, w.G
     n_valid = int(batch["lens"].sum().item())
@@ -236,17 +236,7 @@ def main():
     clocks = sampler.stop()
     launches = trl.trl_kernel_launches() - launches0
     trl.check_status(status)
-    elapsed_ms = t_start.elapsed_time(t_end)
-    if dist is not None:
-        t = torch.tensor([elapsed_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(t.item())
-        tot = torch.tensor([n_valid], device=dev, dtype=torch.int64)
-        dist.all_reduce(tot)
-        total_valid = int(tot.item())
-    else:
-        total_valid = n_valid
-    value = total_valid * args.steps / (elapsed_ms * 1e-3)
+    value, elapsed_ms, total_valid = dp.aggregate_throughput(t_start.elapsed_time(t_end), n_valid, args.steps, dev)
 
     # per-call device times (this rank), averaged over the timed steps
     names = ["token_logprobs_policy", "token_logprobs_old", "hrd_advantages", "pg_loss_fwd", "pg_loss_bwd"]
@@ -273,11 +263,7 @@ def main():
     for _ in range(e2e_steps):
         e2e_step()
     e2e_s = time.perf_counter() - t0
-    if dist is not None:
-        t = torch.tensor([e2e_s], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
-    e2e_value = total_valid * e2e_steps / e2e_s
+    e2e_value, _, _ = dp.aggregate_throughput(1e3 * e2e_s, n_valid, e2e_steps, dev)
 
     # ---- roofline of the dominant kernel: the tcgen05 GEMM with the log-sum-exp epilogue
     # (2 launches per step, 40 % of the executed FLOPs).  Its launch is timed through the

@@ -1,0 +1,280 @@
+"""Full-size parity: the benchmark's shapes and launch configuration, checked on sampled
+outputs the fp64 oracle can compute one by one, on full oracle runs of the cheap steps, and
+on invariants.  All calls go through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import trl_oracle as orc
+from paper_2510_17891_b200 import synth
+from tests._util import f64, rel_fro, TOL_LOGP, TOL_LOSS, TOL_GRAD
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module")
+def trl():
+    import paper_2510_17891_b200 as t
+    t.load_library()
+    return t
+
+
+def sample_rows(w, lens, bnd, n_random=32, n_rollouts=8, seed=0):
+    """Global row indices worth checking: first / last valid row, both sides of the plan/code
+    boundary and of a 128-row block edge for a few rollouts, plus random valid rows."""
+    r = np.random.default_rng(seed)
+    rows = set()
+    for b in r.choice(w.B, size=min(n_rollouts, w.B), replace=False):
+        L, Bd = int(lens[b]), int(bnd[b])
+        if L == 0:
+            continue
+        for t in (0, L - 1, Bd - 1, Bd, 127, 128, (L - 1) // 128 * 128):
+            if 0 <= t < L:
+                rows.add(int(b) * w.T + t)
+    valid = np.nonzero((np.arange(w.T)[None, :] < lens[:, None]).ravel())[0]
+    rows.update(int(x) for x in r.choice(valid, size=min(n_random, valid.size), replace=False))
+    return np.array(sorted(rows))
+
+
+def oracle_rows_logp(hidden, W64, ids, rows):
+    """Oracle logp / lse for the given global rows (each row is independent)."""
+    Hs = f64(hidden[torch.as_tensor(rows, device=hidden.device)])
+    logp, lse = orc.token_logprobs(Hs, W64, ids[rows], np.array([len(rows)]), T=len(rows))
+    return logp, lse
+
+
+@pytest.fixture(scope="module")
+def cfg2_batch():
+    w = synth.CONFIGS[2]
+    batch = synth.make_batch(w, device=DEV)
+    return w, batch
+
+
+def test_config1_forward_scoring_sampled_rows(trl, cfg2_batch):
+    # config 1 = the forward of config 2's shape: policy and old-policy log-probs plus LSE
+    w, batch = cfg2_batch
+    lens, bnd, ids = batch["lens"].cpu().numpy(), batch["bnd"].cpu().numpy(), batch["ids"].cpu().numpy()
+    rows = sample_rows(w, lens, bnd)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    for Wk in ("W", "W_old"):
+        logp, lse = trl.trl_token_logprobs(batch["hidden"], batch[Wk], batch["ids"], batch["lens"], w.T, status=status)
+        torch.cuda.synchronize()
+        trl.check_status(status)
+        ref_logp, ref_lse = oracle_rows_logp(batch["hidden"], f64(batch[Wk]), ids, rows)
+        assert np.abs(f64(logp)[rows] - ref_logp).max() <= TOL_LOGP
+        assert np.abs(f64(lse)[rows] - ref_lse).max() <= TOL_LOGP
+        # padded rows are exactly zero; valid rows are finite and negative
+        valid = torch.arange(w.T, device=DEV)[None, :] < batch["lens"][:, None]
+        lp = logp.view(w.B, w.T)
+        assert not lp[~valid].any() and not lse.view(w.B, w.T)[~valid].any()
+        assert torch.isfinite(lp).all() and (lp[valid] < 0).all()
+
+
+def test_config2_backward_sampled_rows_full_dW(trl, cfg2_batch):
+    """Backward at the benchmark shape with g non-zero on sampled rows only: every other row
+    contributes exactly nothing, so the oracle on the sampled rows gives the complete dW and
+    the sampled rows of dHidden."""
+    w, batch = cfg2_batch
+    lens, bnd, ids = batch["lens"].cpu().numpy(), batch["bnd"].cpu().numpy(), batch["ids"].cpu().numpy()
+    rows = sample_rows(w, lens, bnd, n_random=48, seed=1)
+    W64 = f64(batch["W"])
+    _, ref_lse = oracle_rows_logp(batch["hidden"], W64, ids, rows)
+    r = np.random.default_rng(2)
+    g_rows = (r.standard_normal(len(rows)) * 1e-5).astype(np.float32)
+    lse_in = torch.full((w.N,), 50.0, device=DEV)
+    lse_in[torch.as_tensor(rows, device=DEV)] = torch.tensor(ref_lse, dtype=torch.float32, device=DEV)
+    g_in = torch.zeros(w.N, device=DEV)
+    g_in[torch.as_tensor(rows, device=DEV)] = torch.tensor(g_rows, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    dH, dW = trl.trl_pg_loss_bwd(batch["hidden"], batch["W"], batch["ids"], batch["lens"], lse_in, g_in, w.T,
+                                 status=status)
+    torch.cuda.synchronize()
+    trl.check_status(status)
+    Hs = f64(batch["hidden"][torch.as_tensor(rows, device=DEV)])
+    lse32 = ref_lse.astype(np.float32).astype(np.float64)
+    ref_dH, ref_dW = orc.pg_loss_bwd(Hs, W64, ids[rows], np.array([len(rows)]), lse32, g_rows.astype(np.float64),
+                                     T=len(rows))
+    assert rel_fro(f64(dH[torch.as_tensor(rows, device=DEV)]), ref_dH) <= TOL_GRAD
+    mask = torch.ones(w.N, dtype=torch.bool, device=DEV)
+    mask[torch.as_tensor(rows, device=DEV)] = False
+    assert not dH[mask].any()
+    dW_host = dW.cpu().numpy()
+    num = den = 0.0
+    for v0 in range(0, w.V, 8192):      # chunked to bound host memory
+        d = dW_host[v0:v0 + 8192].astype(np.float64) - ref_dW[v0:v0 + 8192]
+        num += float((d * d).sum()); den += float((ref_dW[v0:v0 + 8192] ** 2).sum())
+    assert (num / den) ** 0.5 <= TOL_GRAD
+    # per-row relative error on rows that matter most: the sampled tokens' own rows and the last vocabulary tile
+    for v in list(ids[rows][:8]) + [0, 127, 128, 255, 256, w.V - 128, w.V - 1]:
+        assert rel_fro(dW_host[v], ref_dW[v]) <= 2 * TOL_GRAD
+
+
+def test_config2_whole_step_sampled_rows_and_invariants(trl, cfg2_batch):
+    """The whole path in the benchmark's launch configuration: log-probs, g and dHidden on
+    sampled rows against a from-scratch oracle per row; integers over all tokens; invariants."""
+    w, batch = cfg2_batch
+    lens, bnd, ids = batch["lens"].cpu().numpy(), batch["bnd"].cpu().numpy(), batch["ids"].cpu().numpy()
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    out = trl.hrd_pg_step(batch, w.P, w.G, w.T, status=status)
+    torch.cuda.synchronize()
+    trl.check_status(status)
+    hrd_ref = orc.hrd_advantages(f64(batch["r_plan"]), f64(batch["r_code"]), lens, bnd, w.P, w.G, w.T)
+    np.testing.assert_array_equal(out["hrd"]["seg"].cpu().numpy(), hrd_ref["seg"])
+    np.testing.assert_array_equal(out["hrd"]["n_plan"].cpu().numpy(), hrd_ref["n_plan"])
+    np.testing.assert_array_equal(out["hrd"]["n_code"].cpu().numpy(), hrd_ref["n_code"])
+    assert int(out["hrd"]["n_valid"].item()) == hrd_ref["n_valid"]
+    np.testing.assert_allclose(f64(out["hrd"]["adv"]), hrd_ref["adv"], rtol=1e-6, atol=1e-7)
+
+    rows = sample_rows(w, lens, bnd, n_random=24, seed=3)
+    W64 = f64(batch["W"])
+    ref_logp, ref_lse = oracle_rows_logp(batch["hidden"], W64, ids, rows)
+    ref_old, _ = oracle_rows_logp(batch["hidden_old"], f64(batch["W_old"]), ids, rows)
+    assert np.abs(f64(out["logp"])[rows] - ref_logp).max() <= TOL_LOGP
+    assert np.abs(f64(out["old_logp"])[rows] - ref_old).max() <= TOL_LOGP
+    # g on the sampled rows from the oracle's own log-probs (row-local given len, adv, P, G)
+    s = np.exp(ref_logp - ref_old)
+    A = hrd_ref["adv"][rows]
+    wgt = np.where(hrd_ref["seg"][rows] == 1, 0.1, 1.0)
+    Lb = lens[rows // w.T]
+    active = A * s <= A * np.clip(s, 0.8, 1.2)
+    ref_g = np.where(active, -wgt * A * s / (w.P * w.G * Lb), 0.0)
+    np.testing.assert_allclose(f64(out["g"])[rows], ref_g, rtol=2e-2, atol=1e-12)
+    # dHidden rows from scratch
+    dH = f64(out["dHidden"][torch.as_tensor(rows, device=DEV)])
+    ref_dH = np.stack([orc.row_dhidden(f64(batch["hidden"][int(n)]), W64, ids[n], ref_g[i]) for i, n in enumerate(rows)])
+    nz = np.linalg.norm(ref_dH, axis=1) > 0
+    assert nz.any()
+    assert rel_fro(dH[nz], ref_dH[nz]) <= TOL_GRAD and not dH[~nz].any()
+    # invariants at full size
+    valid = (torch.arange(w.T, device=DEV)[None, :] < batch["lens"][:, None]).reshape(-1)
+    assert not out["dHidden"][~valid].any() and not out["g"][~valid].any()
+    col = out["dW"].double().sum(dim=0)                         # sum_v dS[n,v] = 0  =>  column sums vanish
+    assert float(col.abs().max()) <= 1e-2 * float(out["dW"].double().abs().sum(dim=0).max())
+    assert torch.isfinite(out["dW"]).all() and torch.isfinite(out["loss"]).all()
+
+
+def test_full_size_advantages_and_loss_all_tokens(trl):
+    """Steps a3 and a4 at the largest token count (config 3: 32 x 8192), every element
+    against the oracle, with generator-made log-probs."""
+    w = synth.CONFIGS[3]
+    g = torch.Generator().manual_seed(7)
+    lens = torch.randint(w.T // 8, w.T + 1, (w.B,), generator=g, dtype=torch.int32)
+    lens[3] = 0
+    bnd = (lens.double() * (torch.rand(w.B, generator=g, dtype=torch.float64) * 0.4 + 0.5)).to(torch.int32)
+    r_plan = (torch.rand(w.B, generator=g) < 0.3).float() * (torch.rand(w.B, generator=g) * 1.8 + 0.2)
+    r_code = (torch.rand(w.B, generator=g) < 0.6).float()
+    old = -torch.rand(w.N, generator=g) * 6
+    logp = old + 0.12 * torch.randn(w.N, generator=g)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    hrd = trl.trl_hrd_advantages(r_plan.to(DEV), r_code.to(DEV), lens.to(DEV), bnd.to(DEV), w.P, w.G, w.T, status=status)
+    loss, gg, stats = trl.trl_pg_loss_fwd(logp.to(DEV), old.to(DEV), hrd["adv"], hrd["seg"], lens.to(DEV), w.P, w.G, w.T,
+                                          status=status)
+    loss2, _, _ = trl.trl_pg_loss_fwd(logp.to(DEV), old.to(DEV), hrd["adv"], hrd["seg"], lens.to(DEV), w.P, w.G, w.T)
+    torch.cuda.synchronize()
+    trl.check_status(status)
+    ref = orc.hrd_advantages(f64(r_plan), f64(r_code), lens.numpy(), bnd.numpy(), w.P, w.G, w.T)
+    np.testing.assert_array_equal(hrd["seg"].cpu().numpy(), ref["seg"])
+    np.testing.assert_array_equal(hrd["n_plan"].cpu().numpy(), ref["n_plan"])
+    np.testing.assert_array_equal(hrd["n_code"].cpu().numpy(), ref["n_code"])
+    assert int(hrd["n_valid"].item()) == ref["n_valid"]
+    np.testing.assert_allclose(f64(hrd["adv"]), ref["adv"], rtol=1e-6, atol=1e-7)
+    rl, rg, rs = orc.pg_loss_fwd(f64(logp), f64(old), ref["adv"], ref["seg"], lens.numpy(), w.P, w.G, w.T)
+    assert abs(float(loss) - rl) <= TOL_LOSS * abs(rl)
+    assert float(loss) == float(loss2)                       # fixed summation order: bit-reproducible
+    assert rel_fro(f64(gg), rg) <= 1e-5
+    np.testing.assert_allclose(f64(stats), rs, rtol=1e-4, atol=1e-6)
+
+
+def test_config3_long_reasoning_whole_step(trl):
+    """Config 3 (32 rollouts x 8192 tokens, heavy padding skew): whole step, sampled rows."""
+    w = synth.CONFIGS[3]
+    batch = synth.make_batch(w, device=DEV)
+    lens, bnd, ids = batch["lens"].cpu().numpy(), batch["bnd"].cpu().numpy(), batch["ids"].cpu().numpy()
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    out = trl.hrd_pg_step(batch, w.P, w.G, w.T, status=status)
+    torch.cuda.synchronize()
+    trl.check_status(status)
+    rows = sample_rows(w, lens, bnd, n_random=16, n_rollouts=6, seed=5)
+    W64 = f64(batch["W"])
+    ref_logp, _ = oracle_rows_logp(batch["hidden"], W64, ids, rows)
+    ref_old, _ = oracle_rows_logp(batch["hidden_old"], f64(batch["W_old"]), ids, rows)
+    assert np.abs(f64(out["logp"])[rows] - ref_logp).max() <= TOL_LOGP
+    hrd_ref = orc.hrd_advantages(f64(batch["r_plan"]), f64(batch["r_code"]), lens, bnd, w.P, w.G, w.T)
+    np.testing.assert_array_equal(out["hrd"]["seg"].cpu().numpy(), hrd_ref["seg"])
+    s = np.exp(ref_logp - ref_old)
+    A = hrd_ref["adv"][rows]
+    wgt = np.where(hrd_ref["seg"][rows] == 1, 0.1, 1.0)
+    active = A * s <= A * np.clip(s, 0.8, 1.2)
+    ref_g = np.where(active, -wgt * A * s / (w.P * w.G * lens[rows // w.T]), 0.0)
+    sel = [i for i in range(len(rows)) if ref_g[i] != 0][:12]
+    assert sel
+    dH = f64(out["dHidden"][torch.as_tensor(rows[sel], device=DEV)])
+    ref_dH = np.stack([orc.row_dhidden(f64(batch["hidden"][int(rows[i])]), W64, ids[rows[i]], ref_g[i]) for i in sel])
+    assert rel_fro(dH, ref_dH) <= TOL_GRAD
+    valid = (torch.arange(w.T, device=DEV)[None, :] < batch["lens"][:, None]).reshape(-1)
+    assert not out["dHidden"][~valid].any()
+
+
+def _sweep_cases():
+    cases = []
+    Gs = (4, 8, 16)
+    k = 0
+    for V in (32000, 65536, 151936, 256000):
+        for H in (2048, 4096, 5120):
+            cases.append((V, H, Gs[k % 3]))
+            k += 1
+    cases += [(65536, 2048, 4), (65536, 2048, 16)]          # all three group sizes at one shape
+    return cases
+
+
+@pytest.mark.parametrize("V,H,G", _sweep_cases())
+def test_config4_shape_sweep(trl, V, H, G):
+    """Config 4: 64 rollouts x T=1024 at each (V, H) with 25 % all-equal reward groups; sampled
+    rows of logp and dHidden and sampled vocabulary rows of dW via the sparse-g backward."""
+    w = synth.Workload(f"cfg4_V{V}_H{H}_G{G}", P=64 // G, G=G, T=1024, H=H, V=V, degenerate_frac=0.25)
+    batch = synth.make_batch(w, device=DEV, with_old_model=False)
+    lens, bnd, ids = batch["lens"].cpu().numpy(), batch["bnd"].cpu().numpy(), batch["ids"].cpu().numpy()
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    logp, lse = trl.trl_token_logprobs(batch["hidden"], batch["W"], batch["ids"], batch["lens"], w.T, status=status)
+    hrd = trl.trl_hrd_advantages(batch["r_plan"], batch["r_code"], batch["lens"], batch["bnd"], w.P, w.G, w.T,
+                                 status=status)
+    old = logp + batch["old_noise"]
+    loss, g, _ = trl.trl_pg_loss_fwd(logp, old, hrd["adv"], hrd["seg"], batch["lens"], w.P, w.G, w.T, status=status)
+    torch.cuda.synchronize()
+    # degenerate groups: advantages, and hence g, are exactly zero on all of their tokens
+    ref = orc.hrd_advantages(f64(batch["r_plan"]), f64(batch["r_code"]), lens, bnd, w.P, w.G, w.T)
+    np.testing.assert_array_equal(hrd["seg"].cpu().numpy(), ref["seg"])
+    np.testing.assert_allclose(f64(hrd["adv"]), ref["adv"], rtol=1e-6, atol=1e-7)
+    assert not g[torch.as_tensor(ref["adv"] == 0, device=DEV)].any()
+    assert (ref["A_plan"].reshape(w.P, w.G) == 0).all(axis=1).sum() >= round(0.25 * w.P)
+
+    rows = sample_rows(w, lens, bnd, n_random=12, n_rollouts=3, seed=V + H + G)
+    W64 = f64(batch["W"])
+    ref_logp, ref_lse = oracle_rows_logp(batch["hidden"], W64, ids, rows)
+    assert np.abs(f64(logp)[rows] - ref_logp).max() <= TOL_LOGP
+    # sparse-g backward
+    r = np.random.default_rng(V + H)
+    g_rows = (r.standard_normal(len(rows)) * 1e-5).astype(np.float32)
+    idx = torch.as_tensor(rows, device=DEV)
+    lse_in = torch.full((w.N,), 50.0, device=DEV)
+    lse_in[idx] = torch.tensor(ref_lse, dtype=torch.float32, device=DEV)
+    g_in = torch.zeros(w.N, device=DEV)
+    g_in[idx] = torch.tensor(g_rows, device=DEV)
+    dH, dW = trl.trl_pg_loss_bwd(batch["hidden"], batch["W"], batch["ids"], batch["lens"], lse_in, g_in, w.T,
+                                 status=status)
+    torch.cuda.synchronize()
+    trl.check_status(status)
+    Hs = f64(batch["hidden"][idx])
+    z = Hs @ W64.T
+    dS = -np.exp(z - ref_lse.astype(np.float32).astype(np.float64)[:, None])
+    dS[np.arange(len(rows)), ids[rows]] += 1.0
+    dS *= g_rows.astype(np.float64)[:, None]
+    assert rel_fro(f64(dH[idx]), dS @ W64) <= TOL_GRAD
+    vsel = np.unique(np.concatenate([ids[rows], [0, 127, 128, 255, 256, V - 129, V - 128, V - 1],
+                                     r.integers(0, V, 64)]))
+    ref_dW_rows = dS[:, vsel].T @ Hs
+    assert rel_fro(f64(dW[torch.as_tensor(vsel, device=DEV)]), ref_dW_rows) <= TOL_GRAD
+    mask = torch.ones(w.N, dtype=torch.bool, device=DEV)
+    mask[idx] = False
+    assert not dH[mask].any()
