@@ -144,6 +144,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", type=int, default=WORKLOAD_ID, help="config number (default: the metric's)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--path", default="fused", choices=["fused", "four_call"],
+                    help="fused: old-policy scoring, advantages, trl_pg_step_fused; four_call: the separate calls")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -181,11 +183,28 @@ def main():
                 old_lse=torch.empty(B * T, **f32), loss=torch.empty(1, **f32), g=torch.empty(B * T, **f32),
                 stats=torch.empty(4, **f32), dHidden=torch.empty_like(batch["hidden"]),
                 dW=torch.empty(V, H, **f32), ws_fwd=ws(trl.TRL_CALL_TOKEN_LOGPROBS),
-                ws_loss=ws(trl.TRL_CALL_PG_LOSS_FWD), ws_bwd=ws(trl.TRL_CALL_PG_LOSS_BWD))
+                ws_loss=ws(trl.TRL_CALL_PG_LOSS_FWD),
+                ws_bwd=ws(trl.TRL_CALL_PG_LOSS_BWD if args.path == "four_call" else trl.TRL_CALL_PG_STEP_FUSED))
+    fused_out = {k: bufs[k] for k in ("logp", "lse", "g", "loss", "stats", "dHidden", "dW")}
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     stream = torch.cuda.current_stream()
 
-    def step(ev=None):
+    def step_fused(ev=None):
+        """One pass: old-policy scoring, HRD advantages, fused policy scoring + loss + backward."""
+        mark = (lambda: None) if ev is None else (lambda: ev.append(_rec()))
+        mark()
+        trl.trl_token_logprobs(batch["hidden_old"], batch["W_old"], batch["ids"], batch["lens"], T, bufs["old_logp"],
+                               bufs["old_lse"], bufs["ws_fwd"], status, stream)
+        mark()
+        hrd = trl.trl_hrd_advantages(batch["r_plan"], batch["r_code"], batch["lens"], batch["bnd"], P, G, T, 0,
+                                     bufs.get("hrd"), status, stream)
+        bufs["hrd"] = hrd
+        mark()
+        trl.trl_pg_step_fused(batch["hidden"], batch["W"], batch["ids"], batch["lens"], bufs["old_logp"], bufs["old_lse"],
+                              hrd["adv"], hrd["seg"], P, G, T, 0.2, 0.2, 0.1, fused_out, bufs["ws_bwd"], status, stream)
+        mark()
+
+    def step_four(ev=None):
         """The five C-ABI calls of one pass.  `ev` collects CUDA events around each call."""
         mark = (lambda: None) if ev is None else (lambda: ev.append(_rec()))
         mark()
@@ -205,6 +224,8 @@ def main():
         trl.trl_pg_loss_bwd(batch["hidden"], batch["W"], batch["ids"], batch["lens"], bufs["lse"], bufs["g"], T,
                             bufs["dHidden"], bufs["dW"], bufs["ws_bwd"], status, stream)
         mark()
+
+    step = step_fused if args.path == "fused" else step_four
 
     def _rec():
         e = torch.cuda.Event(enable_timing=True)
@@ -239,7 +260,8 @@ def main():
     value, elapsed_ms, total_valid = dp.aggregate_throughput(t_start.elapsed_time(t_end), n_valid, args.steps, dev)
 
     # per-call device times (this rank), averaged over the timed steps
-    names = ["token_logprobs_policy", "token_logprobs_old", "hrd_advantages", "pg_loss_fwd", "pg_loss_bwd"]
+    names = (["token_logprobs_old", "hrd_advantages", "pg_step_fused"] if args.path == "fused" else
+             ["token_logprobs_policy", "token_logprobs_old", "hrd_advantages", "pg_loss_fwd", "pg_loss_bwd"])
     call_ms = {n: statistics.mean(ev[i].elapsed_time(ev[i + 1]) for ev in call_events) for i, n in enumerate(names)}
 
     # ---- end-to-end: host buffers in, loss out, copies inside the timed region
@@ -266,16 +288,19 @@ def main():
     e2e_value, _, _ = dp.aggregate_throughput(1e3 * e2e_s, n_valid, e2e_steps, dev)
 
     # ---- roofline of the dominant kernel: the tcgen05 GEMM with the log-sum-exp epilogue
-    # (2 launches per step, 40 % of the executed FLOPs).  Its launch is timed through the
+    # (the largest single launch of the step).  Its launch is timed through the
     # trl_token_logprobs call that contains it (plus two sub-millisecond helper kernels).
     flops_fwd = 2.0 * H * V * n_valid
-    t_fwd_ms = 0.5 * (call_ms["token_logprobs_policy"] + call_ms["token_logprobs_old"])
+    t_fwd_ms = call_ms["token_logprobs_old"]
     achieved = flops_fwd / (t_fwd_ms * 1e-3) / 1e12
     peak = peaks["bf16_sustained"]
     roofline = dict(bound="tensor", kernel="tc_gemm_kernel<LSE> (inside trl_token_logprobs)", achieved=achieved,
                     peak=peak, unit="TFLOP/s", frac=achieved / peak, traffic=None,
                     peak_source=f"{peaks['source']} sustained cuBLAS bf16")
-    bwd_alg = 4.0 * H * V * n_valid / (call_ms["pg_loss_bwd"] * 1e-3) / 1e12
+    if args.path == "fused":     # policy forward + two gradient GEMMs = the metric's 6HV per token
+        rest_alg = 6.0 * H * V * n_valid / (call_ms["pg_step_fused"] * 1e-3) / 1e12
+    else:
+        rest_alg = 4.0 * H * V * n_valid / (call_ms["pg_loss_bwd"] * 1e-3) / 1e12
     step_alg = 6.0 * H * V * value / world / 1e12
 
     cpu_baseline = None
@@ -296,7 +321,8 @@ def main():
                                                note="6*H*V FLOP per scored token over the whole step (which also scores the old policy)"),
                     roofline=roofline,
                     calls_ms=call_ms,
-                    bwd_algorithmic_tflops=bwd_alg,
+                    path=args.path,
+                    algorithmic_tflops_of_last_call=rest_alg,
                     e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
                              steps=e2e_steps),
                     gpu_launches=int(launches),

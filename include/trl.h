@@ -49,7 +49,8 @@ typedef enum {
   TRL_ERR_ARCH = 5,       /* device is not compute capability 10.x */
   TRL_ERR_CUDA = 6,       /* a CUDA runtime / driver call failed   */
   TRL_ERR_BAD_INDEX = 7,  /* device-detected: id, len or bnd out of range */
-  TRL_ERR_TIMEOUT = 8     /* device-detected: a bounded pipeline wait expired */
+  TRL_ERR_TIMEOUT = 8,    /* device-detected: a bounded pipeline wait expired */
+  TRL_ERR_BAD_HINT = 9    /* device-detected: lse_hint so far off that exp(z - hint) left the fp32 range */
 } trl_status;
 
 /* Storage type of hidden / W / dHidden.  TRL_BF16 runs on the tcgen05 tensor cores with
@@ -59,7 +60,8 @@ typedef enum { TRL_F32 = 0, TRL_BF16 = 1 } trl_dtype;
 typedef enum {
   TRL_CALL_TOKEN_LOGPROBS = 0,
   TRL_CALL_PG_LOSS_FWD = 1,
-  TRL_CALL_PG_LOSS_BWD = 2
+  TRL_CALL_PG_LOSS_BWD = 2,
+  TRL_CALL_PG_STEP_FUSED = 3
 } trl_call;
 
 /* Hyper-parameters of the surrogate.  The paper uses eps_lo = eps_hi = 0.2 (training
@@ -156,6 +158,33 @@ int trl_pg_loss_bwd(const void* hidden, const void* W, const int32_t* ids, const
                     int B, int T, int H, int V, trl_dtype dt,
                     void* dHidden, float* dW,
                     void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream);
+
+/*
+ * Fused schedule of trl_token_logprobs (current policy) + trl_pg_loss_fwd + trl_pg_loss_bwd:
+ * same inputs, same outputs, same definitions (Section 2.3 objective and its chain rule), but
+ * the forward GEMM is not repeated in the backward.  Per chunk of rows the forward GEMM stores
+ * E = exp(z - c) (bf16, chunk-bounded scratch) for a per-row shift c = lse_hint[n]; then
+ * lse = c + log sum_v E, logp, g follow per row, and because softmax = E exp(c - lse) the
+ * gradient GEMMs run on E directly with the per-row factor folded into their other operand.
+ * Results do not depend on c beyond rounding.
+ *
+ * lse_hint [B*T] f32: any value within ~80 of the row's true log-partition, e.g. the old
+ * policy's lse from trl_token_logprobs.  NULL: the exact lse is computed first by an extra
+ * forward pass (then this call costs what the three separate calls cost).  A hint so wrong that
+ * exp(z - hint) overflows sets TRL_ERR_BAD_HINT in *status_dev.
+ *
+ * in : hidden, W, ids, len as in trl_token_logprobs; old_logp, adv [B*T] f32, seg [B*T] u8
+ *      (from trl_hrd_advantages); lse_hint or NULL
+ * out: logp, lse, g [B*T] f32 (0 on padding); loss [1]; stats [4] or NULL;
+ *      dHidden [B*T,H] dt (padded rows 0); dW [V,H] f32 (overwritten)
+ * TRL_F32 runs the three separate calls internally.
+ */
+int trl_pg_step_fused(const void* hidden, const void* W, const int32_t* ids, const int32_t* len,
+                      const float* old_logp, const float* lse_hint, const float* adv, const uint8_t* seg,
+                      int P, int G, int T, int H, int V, trl_dtype dt, trl_pg_config cfg,
+                      float* logp, float* lse, float* loss, float* g, float* stats,
+                      void* dHidden, float* dW,
+                      void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream);
 
 /*
  * Same computation and outputs as trl_pg_loss_fwd, for callers that cannot allocate device

@@ -5,8 +5,9 @@ import os
 import torch
 
 TRL_F32, TRL_BF16 = 0, 1
-TRL_CALL_TOKEN_LOGPROBS, TRL_CALL_PG_LOSS_FWD, TRL_CALL_PG_LOSS_BWD = 0, 1, 2
-_STATUS_BITS = {7: "index out of range (token id / len / bnd)", 8: "pipeline wait timed out"}
+TRL_CALL_TOKEN_LOGPROBS, TRL_CALL_PG_LOSS_FWD, TRL_CALL_PG_LOSS_BWD, TRL_CALL_PG_STEP_FUSED = 0, 1, 2, 3
+_STATUS_BITS = {7: "index out of range (token id / len / bnd)", 8: "pipeline wait timed out",
+                9: "lse_hint out of range"}
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
 _lib = None
@@ -35,6 +36,7 @@ _SIGNATURES = {
     "trl_hrd_advantages": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "trl_pg_loss_fwd": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, PgConfig, _vp, _vp, _vp, _vp, _sz, _vp, _vp]),
     "trl_pg_loss_fwd_static": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, PgConfig, _vp, _vp, _vp, _vp, _vp]),
+    "trl_pg_step_fused": (_i, [_vp] * 8 + [_i] * 6 + [PgConfig] + [_vp] * 7 + [_vp, _sz, _vp, _vp]),
     "trl_pg_loss_bwd": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _vp, _vp, _sz, _vp, _vp]),
 }
 
@@ -208,12 +210,53 @@ def trl_pg_loss_bwd(hidden, W, ids, lens, lse, g, T, dHidden=None, dW=None, work
     return dHidden, dW
 
 
+def trl_pg_step_fused(hidden, W, ids, lens, old_logp, lse_hint, adv, seg, P, G, T, eps_lo=0.2, eps_hi=0.2, alpha=0.1,
+                      out=None, workspace=None, status=None, stream=None):
+    """Fused policy scoring + surrogate loss + backward (see include/trl.h).  `lse_hint` may be
+    None.  Returns a dict with logp, lse, loss, g, stats, dHidden, dW."""
+    _dev(hidden, W, ids, lens, old_logp, lse_hint, adv, seg, workspace, status)
+    B = lens.numel()
+    V, H = W.shape
+    dt = _dt(hidden)
+    dev = hidden.device
+    o = {} if out is None else out
+    f32 = dict(dtype=torch.float32, device=dev)
+    for k, shape in (("logp", B * T), ("lse", B * T), ("g", B * T), ("loss", 1), ("stats", 4)):
+        if o.get(k) is None:
+            o[k] = torch.empty(shape, **f32)
+    if o.get("dHidden") is None:
+        o["dHidden"] = torch.empty_like(hidden)
+    if o.get("dW") is None:
+        o["dW"] = torch.empty(V, H, **f32)
+    if workspace is None:
+        workspace = _workspace(trl_workspace_bytes(TRL_CALL_PG_STEP_FUSED, B, T, H, V, dt), dev)
+    rc = load_library().trl_pg_step_fused(_ptr(hidden), _ptr(W), _ptr(ids), _ptr(lens), _ptr(old_logp), _ptr(lse_hint),
+                                          _ptr(adv), _ptr(seg), P, G, T, H, V, dt, PgConfig(eps_lo, eps_hi, alpha),
+                                          _ptr(o["logp"]), _ptr(o["lse"]), _ptr(o["loss"]), _ptr(o["g"]),
+                                          _ptr(o["stats"]), _ptr(o["dHidden"]), _ptr(o["dW"]), _ptr(workspace),
+                                          workspace.numel(), _ptr(status), _stream(stream))
+    _check(rc, "trl_pg_step_fused")
+    return o
+
+
 def hrd_pg_step(batch, P, G, T, eps_lo=0.2, eps_hi=0.2, alpha=0.1, adv_mode=0, old_logp=None, bufs=None,
-                status=None, stream=None):
+                status=None, stream=None, fused=False, use_hint=True):
     """One pass of the whole path by calling the five C entry points in order: score under the
     current and the old policy, HRD advantages, surrogate loss, backward.  `bufs` may carry
     preallocated outputs / workspaces (keys as returned).  No arithmetic happens here."""
     bufs = {} if bufs is None else bufs
+    if fused:
+        old_lse = None
+        if old_logp is None:
+            old_logp, old_lse = trl_token_logprobs(batch["hidden_old"], batch["W_old"], batch["ids"], batch["lens"], T,
+                                                   bufs.get("old_logp"), bufs.get("old_lse"), bufs.get("ws_fwd"),
+                                                   status, stream)
+        hrd = trl_hrd_advantages(batch["r_plan"], batch["r_code"], batch["lens"], batch["bnd"], P, G, T, adv_mode,
+                                 bufs.get("hrd"), status, stream)
+        o = trl_pg_step_fused(batch["hidden"], batch["W"], batch["ids"], batch["lens"], old_logp,
+                              old_lse if use_hint else None, hrd["adv"], hrd["seg"], P, G, T, eps_lo, eps_hi, alpha,
+                              bufs.get("fused_out"), bufs.get("ws_fused"), status, stream)
+        return dict(old_logp=old_logp, hrd=hrd, **o)
     logp, lse = trl_token_logprobs(batch["hidden"], batch["W"], batch["ids"], batch["lens"], T,
                                    bufs.get("logp"), bufs.get("lse"), bufs.get("ws_fwd"), status, stream)
     if old_logp is None:

@@ -52,6 +52,12 @@ size_t bwd_bytes_f32(int B, int T, int H, int V, int R) {
   return row_blocks_bytes(B, T) + 2 * align_up((size_t)R * H * 4, 256) + align_up((size_t)R * V * 4, 256);
 }
 int rows_cap_of(int B, int T) { return B * cdiv(T, kRowBlock) * kRowBlock; }
+size_t loss_bytes(int B, int T) { return align_up((size_t)B * pg_loss_tiles(T) * 4 * sizeof(float), 256); }
+// fused step: fixed part (row blocks, W^T, loss partials) and per-chunk part for R rows
+size_t fused_fixed_bf16(int B, int T, int H, int V) { return bwd_fixed_bf16(B, T, H, V) + loss_bytes(B, T); }
+size_t fused_per_rows_bf16(int H, int V, int R) {
+  return bwd_per_rows_bf16(H, V, R) + align_up((size_t)cdiv(V, 256) * R * 4, 256) + 2 * align_up((size_t)R * 4, 256);
+}
 
 // largest multiple of 128 rows (<= cap) whose scratch fits into `avail` bytes
 template <class F>
@@ -80,6 +86,17 @@ size_t ws_bytes(int which, int B, int T, int H, int V, trl_dtype dt, bool minimu
         return bwd_fixed_bf16(B, T, H, V) + bwd_per_rows_bf16(H, V, R);
       }
       return bwd_bytes_f32(B, T, H, V, minimum ? kRowBlock : (cap < kRecommendedChunkRowsF32 ? cap : kRecommendedChunkRowsF32));
+    case TRL_CALL_PG_STEP_FUSED: {
+      if (dt == TRL_BF16) {
+        const int R = minimum ? kRowBlock : (cap < kRecommendedChunkRowsBf16 ? cap : kRecommendedChunkRowsBf16);
+        // the forward workspace is appended for the lse_hint == NULL case
+        return fused_fixed_bf16(B, T, H, V) + fused_per_rows_bf16(H, V, R) + fwd_bytes_bf16(B, T, V);
+      }
+      size_t a = ws_bytes(TRL_CALL_TOKEN_LOGPROBS, B, T, H, V, dt, minimum);
+      size_t b = ws_bytes(TRL_CALL_PG_LOSS_BWD, B, T, H, V, dt, minimum);
+      size_t c = loss_bytes(B, T);
+      return (a > b ? a : b) > c ? (a > b ? a : b) : c;
+    }
   }
   return 0;
 }
@@ -110,6 +127,7 @@ const char* trl_status_string(int status) {
     case TRL_ERR_CUDA: return "CUDA error";
     case TRL_ERR_BAD_INDEX: return "index out of range (device)";
     case TRL_ERR_TIMEOUT: return "pipeline wait timed out (device)";
+    case TRL_ERR_BAD_HINT: return "lse_hint out of range (device)";
   }
   return "unknown status";
 }
@@ -225,7 +243,7 @@ int trl_pg_loss_bwd(const void* hidden, const void* W, const int32_t* ids, const
     launch_transpose_bf16((const __nv_bfloat16*)W, Wt, V, H, s);
     const int CB = R / kRowBlock;
     for (int blk_off = 0; blk_off < rb.cap; blk_off += CB) {
-      launch_gather_transpose_bf16((const __nv_bfloat16*)hidden, Xt, H, R, rb, blk_off, s);
+      launch_gather_transpose_bf16((const __nv_bfloat16*)hidden, Xt, H, R, rb, blk_off, nullptr, s);
       TcGemm a;
       memset(&a, 0, sizeof(a));
       a.rb = rb; a.blk_off = blk_off; a.blk_cap = CB; a.status = status_dev;
@@ -270,6 +288,110 @@ int trl_pg_loss_bwd(const void* hidden, const void* W, const int32_t* ids, const
       launch_simt_gemm(dw, s);
     }
   }
+  TRL_CUDA_OK(cudaGetLastError());
+  return TRL_OK;
+}
+
+
+int trl_pg_step_fused(const void* hidden, const void* W, const int32_t* ids, const int32_t* len,
+                      const float* old_logp, const float* lse_hint, const float* adv, const uint8_t* seg,
+                      int P, int G, int T, int H, int V, trl_dtype dt, trl_pg_config cfg,
+                      float* logp, float* lse, float* loss, float* g, float* stats, void* dHidden, float* dW,
+                      void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream) {
+  if (!hidden || !W || !ids || !len || !old_logp || !adv || !seg || !logp || !lse || !loss || !g || !dHidden || !dW ||
+      !workspace)
+    return TRL_ERR_INVALID_ARG;
+  if (dt != TRL_F32 && dt != TRL_BF16) return TRL_ERR_DTYPE;
+  if (P <= 0 || G <= 0 || (long)P * G > 65535) return TRL_ERR_SHAPE;
+  const int B = P * G;
+  if (!shapes_ok(B, T, H, V)) return TRL_ERR_SHAPE;
+  if (dt == TRL_BF16 && ((H % 8) || (V % 8))) return TRL_ERR_SHAPE;
+  if (!(cfg.eps_lo >= 0.f) || !(cfg.eps_hi >= 0.f) || !(cfg.alpha >= 0.f)) return TRL_ERR_INVALID_ARG;
+  if (((uintptr_t)workspace & 255) != 0) return TRL_ERR_INVALID_ARG;
+  if (workspace_bytes < trl_workspace_bytes_min(TRL_CALL_PG_STEP_FUSED, B, T, H, V, dt)) return TRL_ERR_WORKSPACE_TOO_SMALL;
+  if (int e = check_device()) return e;
+
+  if (dt == TRL_F32) {   // the fp32 path has no fused schedule: run the three calls in order
+    if (int e = trl_token_logprobs(hidden, W, ids, len, B, T, H, V, dt, logp, lse, workspace, workspace_bytes, status_dev, stream)) return e;
+    if (int e = trl_pg_loss_fwd(logp, old_logp, adv, seg, len, P, G, T, cfg, loss, g, stats, workspace, workspace_bytes, status_dev, stream)) return e;
+    return trl_pg_loss_bwd(hidden, W, ids, len, lse, g, B, T, H, V, dt, dHidden, dW, workspace, workspace_bytes, status_dev, stream);
+  }
+
+  cudaStream_t s = (cudaStream_t)stream;
+  const int cap_rows = rows_cap_of(B, T);
+  const size_t N = (size_t)B * T;
+  const int nt = cdiv(V, 256);
+  const size_t fwd_extra = lse_hint ? 0 : fwd_bytes_bf16(B, T, V);
+  if (workspace_bytes < fused_fixed_bf16(B, T, H, V) + fwd_extra + fused_per_rows_bf16(H, V, kRowBlock))
+    return TRL_ERR_WORKSPACE_TOO_SMALL;
+  const size_t avail = workspace_bytes - fused_fixed_bf16(B, T, H, V) - fwd_extra;
+  const int R = fit_rows(avail, cap_rows < kRecommendedChunkRowsBf16 ? cap_rows : kRecommendedChunkRowsBf16,
+                         [&](int r) { return fused_per_rows_bf16(H, V, r); });
+  if (R < kRowBlock) return TRL_ERR_WORKSPACE_TOO_SMALL;
+
+  Carver cv(workspace);
+  RowBlocks rb = carve_row_blocks(cv.take<char>(row_blocks_bytes(B, T)), B, T);
+  __nv_bfloat16* Wt = cv.take<__nv_bfloat16>((size_t)H * V);
+  float* loss_partials = cv.take<float>((size_t)B * pg_loss_tiles(T) * 4);
+  __nv_bfloat16* Xt = cv.take<__nv_bfloat16>((size_t)H * R);
+  __nv_bfloat16* E = cv.take<__nv_bfloat16>((size_t)R * V);
+  __nv_bfloat16* Et = cv.take<__nv_bfloat16>((size_t)V * R);
+  float* psum = cv.take<float>((size_t)nt * R);
+  float* tgt = cv.take<float>(R);
+  float* neg_alpha = cv.take<float>(R);
+
+  launch_build_row_blocks(len, B, T, rb, status_dev, s);
+  TRL_CUDA_OK(cudaMemsetAsync(dW, 0, (size_t)V * H * sizeof(float), s));
+  TRL_CUDA_OK(cudaMemsetAsync(dHidden, 0, N * H * 2, s));
+  launch_zero_padded_f32(logp, lse, len, B, T, s);
+
+  TcGemm base;
+  memset(&base, 0, sizeof(base));
+  base.rb = rb; base.status = status_dev;
+
+  const float* hint = lse_hint;
+  if (!hint) {   // exact log-partition first; it then serves as the shift, so E is the softmax itself
+    float* tgt_all = cv.take<float>(cap_rows);
+    float2* partials = cv.take<float2>((size_t)nt * cap_rows);
+    TcGemm f = base;
+    f.epi = TC_EPI_LSE; f.raster_band = kRasterBandFwd;
+    f.A = hidden; f.a_rows = (long)N; f.a_ld = H; f.B = W; f.b_rows = V; f.b_ld = H; f.K = H; f.N = V;
+    f.blk_off = 0; f.blk_cap = rb.cap; f.ids = ids; f.partials = partials; f.tgt = tgt_all; f.rows_cap = cap_rows;
+    TRL_CUDA_OK(launch_tc_gemm(f, s));
+    launch_merge_lse(partials, tgt_all, nt, cap_rows, rb, ids, len, B, T, V, logp, lse, status_dev, s);
+    hint = lse;
+  }
+
+  launch_transpose_bf16((const __nv_bfloat16*)W, Wt, V, H, s);
+  const int CB = R / kRowBlock;
+  for (int blk_off = 0; blk_off < rb.cap; blk_off += CB) {
+    TcGemm a = base;
+    a.blk_off = blk_off; a.blk_cap = CB;
+    // forward tile -> E = exp(z - c), row sums, sampled token's logit
+    TcGemm e = a;
+    e.epi = TC_EPI_E; e.raster_band = kRasterBandFwd;
+    e.A = hidden; e.a_rows = (long)N; e.a_ld = H; e.B = W; e.b_rows = V; e.b_ld = H; e.K = H; e.N = V;
+    e.ids = ids; e.lse = hint; e.dS = E; e.ds_ld = V; e.dSt = Et; e.dst_ld = R; e.psum = psum; e.tgt = tgt; e.rows_cap = R;
+    TRL_CUDA_OK(launch_tc_gemm(e, s));
+    FusedMergeArgs m{psum, tgt, nt, R, rb, blk_off, ids, len, hint, old_logp, adv, seg, P, G, T, V, cfg,
+                     logp, lse, g, neg_alpha, E, Et, status_dev};
+    launch_fused_merge(m, s);
+    launch_gather_transpose_bf16((const __nv_bfloat16*)hidden, Xt, H, R, rb, blk_off, neg_alpha, s);
+    // dHidden rows = neg_alpha * (E' W)
+    TcGemm dh = a;
+    dh.epi = TC_EPI_DH; dh.raster_band = kRasterBandBwd;
+    dh.A = E; dh.a_rows = R; dh.a_ld = V; dh.B = Wt; dh.b_rows = H; dh.b_ld = V; dh.K = V; dh.N = H;
+    dh.dHidden = (__nv_bfloat16*)dHidden; dh.dh_ld = H; dh.row_scale = neg_alpha;
+    TRL_CUDA_OK(launch_tc_gemm(dh, s));
+    // dW += E'^T (neg_alpha * hidden)
+    TcGemm dw = a;
+    dw.epi = TC_EPI_DW; dw.raster_band = kRasterBandBwd;
+    dw.A = Et; dw.a_rows = V; dw.a_ld = R; dw.B = Xt; dw.b_rows = H; dw.b_ld = R; dw.K = R; dw.N = H;
+    dw.m_blocks = cdiv(V, kRowBlock); dw.dW = dW; dw.dw_ld = H; dw.V = V;
+    TRL_CUDA_OK(launch_tc_gemm(dw, s));
+  }
+  // loss, statistics (and g once more, identically) over all rows now that logp is complete
+  launch_pg_loss(logp, old_logp, adv, seg, len, P, G, T, cfg, loss, g, stats, loss_partials, s);
   TRL_CUDA_OK(cudaGetLastError());
   return TRL_OK;
 }

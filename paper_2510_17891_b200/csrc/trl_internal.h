@@ -46,8 +46,20 @@ void launch_merge_lse(const float2* partials, const float* tgt, int n_tiles, int
                       int32_t* status, cudaStream_t s);
 void launch_transpose_bf16(const __nv_bfloat16* in, __nv_bfloat16* out, int rows, int cols, cudaStream_t s);
 // Xt[h, r] = hidden[row(blk_off*128 + r), h] for the live rows of a chunk, 0 elsewhere
+// (times col_scale[r] when given)
 void launch_gather_transpose_bf16(const __nv_bfloat16* hidden, __nv_bfloat16* Xt, int H, int R, RowBlocks rb,
-                                  int blk_off, cudaStream_t s);
+                                  int blk_off, const float* col_scale, cudaStream_t s);
+// Chunk-local finish of the fused step: lse = c + log(sum_k psum), logp, g = d loss/d logp,
+// the per-row factor -g exp(c - lse) for the gradient GEMMs, and the one-hot fix of E / E^T.
+struct FusedMergeArgs {
+  const float* psum; const float* tgt; int n_tiles; int R; RowBlocks rb; int blk_off;
+  const int32_t* ids; const int32_t* len; const float* hint; const float* old_logp; const float* adv;
+  const uint8_t* seg; int P, G, T, V; trl_pg_config cfg;
+  float* logp; float* lse; float* g; float* neg_alpha;
+  __nv_bfloat16* E; __nv_bfloat16* Et;
+  int32_t* status;
+};
+void launch_fused_merge(const FusedMergeArgs& a, cudaStream_t s);
 // fp32 path helpers
 void launch_pack_rows_f32(const float* hidden, float* Xp, int H, int R, RowBlocks rb, int blk_off, cudaStream_t s);
 void launch_row_lse_f32(const float* S, int V, int R, RowBlocks rb, int blk_off, const int32_t* ids,
@@ -72,7 +84,7 @@ struct SimtGemm {
 void launch_simt_gemm(const SimtGemm& p, cudaStream_t s);
 
 // ---- tcgen05 GEMM family (trl_tc_gemm.cu) ------------------------------------------
-enum TcEpilogue { TC_EPI_LSE = 0, TC_EPI_DS = 1, TC_EPI_DH = 2, TC_EPI_DW = 3 };
+enum TcEpilogue { TC_EPI_LSE = 0, TC_EPI_DS = 1, TC_EPI_DH = 2, TC_EPI_DW = 3, TC_EPI_E = 4 };
 struct TcGemm {
   int epi;
   // operands: A [a_rows, K] and B [b_rows, K], both bf16 row-major with K contiguous
@@ -89,6 +101,8 @@ struct TcGemm {
   __nv_bfloat16* dS; long ds_ld; __nv_bfloat16* dSt; long dst_ld;   // DS
   __nv_bfloat16* dHidden; long dh_ld;                  // DH
   float* dW; long dw_ld; int V;                        // DW
+  float* psum;                                         // E: row sums per vocabulary tile [n_tiles, rows_cap]
+  const float* row_scale;                              // DH: optional per-scratch-row factor
   int32_t* status;
 };
 // returns cudaSuccess or the error of tensor-map creation / launch

@@ -338,7 +338,8 @@ void launch_transpose_bf16(const __nv_bfloat16* in, __nv_bfloat16* out, int rows
 // Xt [H, R]: column r is hidden row (block blk_off + r/128, lane r%128) or 0 if not live.
 __global__ void __launch_bounds__(256) gather_transpose_bf16_kernel(const __nv_bfloat16* __restrict__ hidden,
                                                                     __nv_bfloat16* __restrict__ Xt, int H, int R,
-                                                                    RowBlocks rb, int blk_off) {
+                                                                    RowBlocks rb, int blk_off,
+                                                                    const float* __restrict__ col_scale) {
   __shared__ __nv_bfloat16 tile[64][66];
   const int r0 = blockIdx.y * 64, h0 = blockIdx.x * 64;     // r0: scratch row, 64 | 128 so one block per tile
   const int blk = blk_off + r0 / kRowBlock;
@@ -349,7 +350,9 @@ __global__ void __launch_bounds__(256) gather_transpose_bf16_kernel(const __nv_b
   for (int i = ty; i < 64; i += 4) {
     const int lr = (r0 % kRowBlock) + i;
     const int h = h0 + tx;
-    tile[i][tx] = (lr < nvalid && h < H) ? hidden[(size_t)(grow0 + lr) * H + h] : __float2bfloat16(0.f);
+    __nv_bfloat16 x = (lr < nvalid && h < H) ? hidden[(size_t)(grow0 + lr) * H + h] : __float2bfloat16(0.f);
+    if (col_scale && lr < nvalid) x = __float2bfloat16_rn(__bfloat162float(x) * col_scale[r0 + i]);
+    tile[i][tx] = x;
   }
   __syncthreads();
   for (int i = ty; i < 64; i += 4) {
@@ -359,9 +362,61 @@ __global__ void __launch_bounds__(256) gather_transpose_bf16_kernel(const __nv_b
 }
 
 void launch_gather_transpose_bf16(const __nv_bfloat16* hidden, __nv_bfloat16* Xt, int H, int R, RowBlocks rb,
-                                  int blk_off, cudaStream_t s) {
+                                  int blk_off, const float* col_scale, cudaStream_t s) {
   dim3 grid(cdiv(H, 64), cdiv(R, 64));
-  gather_transpose_bf16_kernel<<<grid, 256, 0, s>>>(hidden, Xt, H, R, rb, blk_off);
+  gather_transpose_bf16_kernel<<<grid, 256, 0, s>>>(hidden, Xt, H, R, rb, blk_off, col_scale);
+  note_launch();
+}
+
+// ------------------------------------------------------------------------------------
+// Fused step, per chunk: one thread per scratch row.  With E = exp(z - c) stored by the GEMM,
+//   lse = c + log sum_v E,  logp = z[id] - lse,  g = d loss / d logp (same formula as
+//   pg_loss_stage1_kernel),  dS = g onehot - g exp(c - lse) E = neg_alpha (E - exp(lse - c) onehot),
+// so the kernel stores neg_alpha = -g exp(c - lse) and subtracts exp(lse - c) from the
+// sampled token's entry of E and E^T.
+// ------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(128) fused_merge_kernel(FusedMergeArgs a) {
+  const int r = blockIdx.x * 128 + threadIdx.x;
+  if (r >= a.R) return;
+  const int blk = a.blk_off + r / kRowBlock;
+  if (blk >= a.rb.nblk[0]) return;
+  const int lr = r % kRowBlock;
+  if (lr >= a.rb.blk_n[blk]) { a.neg_alpha[r] = 0.f; return; }
+  const size_t n = (size_t)a.rb.blk_row[blk] + lr;
+  const int b = (int)(n / a.T);
+  float sum = 0.f;
+  for (int k = 0; k < a.n_tiles; ++k) sum += a.psum[(size_t)k * a.R + r];
+  const float c = a.hint[n];
+  const float lse = c + logf(sum);
+  const int id = a.ids[n];
+  const bool id_ok = (unsigned)id < (unsigned)a.V;
+  if (!id_ok) flag_status(a.status, TRL_ERR_BAD_INDEX);
+  if (!(sum > 0.f) || !isfinite(sum)) flag_status(a.status, TRL_ERR_BAD_HINT);
+  const float lp = id_ok ? a.tgt[r] - lse : 0.f;
+  a.logp[n] = lp;
+  a.lse[n] = lse;
+  const int L = max(0, min(a.len[b], a.T));
+  const float inv = 1.0f / ((float)a.P * (float)a.G * (float)L);
+  const float s = expf(lp - a.old_logp[n]);
+  const float A = a.adv[n];
+  const int sg = a.seg[n];
+  const float w = sg == 1 ? a.cfg.alpha : (sg == 2 ? 1.0f : 0.f);
+  const float unclipped = A * s;
+  const float clipped = A * fminf(fmaxf(s, 1.0f - a.cfg.eps_lo), 1.0f + a.cfg.eps_hi);
+  const float gn = (id_ok && unclipped <= clipped) ? -w * A * s * inv : 0.f;
+  a.g[n] = gn;
+  a.neg_alpha[r] = -gn * expf(c - lse);
+  if (gn != 0.f) {
+    const float beta = expf(lse - c);
+    __nv_bfloat16* e = a.E + (size_t)r * a.V + id;
+    const __nv_bfloat16 fixed = __float2bfloat16_rn(__bfloat162float(*e) - beta);
+    *e = fixed;
+    a.Et[(size_t)id * a.R + r] = fixed;
+  }
+}
+
+void launch_fused_merge(const FusedMergeArgs& a, cudaStream_t s) {
+  fused_merge_kernel<<<cdiv(a.R, 128), 128, 0, s>>>(a);
   note_launch();
 }
 

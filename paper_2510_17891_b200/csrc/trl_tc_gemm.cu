@@ -8,6 +8,10 @@
 //   DS  : dS = g (onehot - exp(z - lse)) as bf16, written row-major and transposed
 //   DH  : dHidden rows (bf16), scattered to the caller's row positions
 //   DW  : dW += tile (fp32 read-modify-write)
+//   E   : E = exp(z - c) for a per-row shift c (a stale log-partition), as bf16 row-major
+//         and transposed, plus the row sums of E and the sampled token's logit.  The softmax
+//         is p = E exp(c - lse), a per-row factor the gradient GEMMs fold into their other
+//         operand / their epilogue, so the forward GEMM is not repeated in the backward.
 //
 // Roles: warp 0 = TMA producer (one elected lane), warp 1 = MMA issuer (one elected lane)
 // and TMEM owner, warps 2..5 = epilogue (one TMEM lane quadrant each).  Shared-memory
@@ -39,6 +43,7 @@ struct TcArgs {
   __nv_bfloat16* dS; long ds_ld; __nv_bfloat16* dSt; long dst_ld;
   __nv_bfloat16* dHidden; long dh_ld;
   float* dW; long dw_ld;
+  float* psum; const float* row_scale;
   int32_t* status;
 };
 
@@ -236,10 +241,57 @@ __device__ __forceinline__ void epilogue_tile(const TcArgs& p, uint32_t tmem_acc
       for (int j = 0; j < 32; ++j)
         if (j < ncl) dst_col[(size_t)j * p.dst_ld] = __float2bfloat16_rn(d[j]);
     }
+  } else if constexpr (EPI == TC_EPI_E) {
+    const int blk = p.blk_off + mb;
+    const bool valid = r < p.blk_n[blk];
+    const long grow = (long)p.blk_row[blk] + r;
+    const int id = valid ? p.ids[grow] : -1;
+    const float C2 = valid ? p.lse[grow] * LOG2E : 0.f;      // p.lse holds the shift c here
+    const size_t srow = (size_t)mb * BM + r;
+    __nv_bfloat16* e_row = p.dS + srow * p.ds_ld;
+    float sum = 0.f, tg = 0.f;
+    bool has = false;
+    for (int c0 = 0; c0 < BN; c0 += 32) {
+      const int ncl = p.N - (n0 + c0);
+      if (ncl <= 0) break;
+      tc_ld32(taddr + c0, v);
+      tc_wait_ld();
+      float d[32];
+#pragma unroll
+      for (int j = 0; j < 32; ++j) {
+        const float e = ex2(fmaf(__uint_as_float(v[j]), LOG2E, -C2));
+        d[j] = (valid && j < ncl) ? e : 0.f;
+        sum += d[j];
+      }
+      const int lc = id - (n0 + c0);
+      if (lc >= 0 && lc < 32 && lc < ncl) {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) if (j == lc) tg = __uint_as_float(v[j]);
+        has = true;
+      }
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        if (q * 8 < ncl) {
+          uint4 w;
+          w.x = pack_bf16x2(d[q * 8 + 0], d[q * 8 + 1]);
+          w.y = pack_bf16x2(d[q * 8 + 2], d[q * 8 + 3]);
+          w.z = pack_bf16x2(d[q * 8 + 4], d[q * 8 + 5]);
+          w.w = pack_bf16x2(d[q * 8 + 6], d[q * 8 + 7]);
+          *reinterpret_cast<uint4*>(e_row + n0 + c0 + q * 8) = w;
+        }
+      }
+      __nv_bfloat16* et_col = p.dSt + (size_t)(n0 + c0) * p.dst_ld + srow;
+#pragma unroll
+      for (int j = 0; j < 32; ++j)
+        if (j < ncl) et_col[(size_t)j * p.dst_ld] = __float2bfloat16_rn(d[j]);
+    }
+    p.psum[(size_t)nt * p.rows_cap + srow] = sum;
+    if (has) p.tgt[srow] = tg;
   } else if constexpr (EPI == TC_EPI_DH) {
     const int blk = p.blk_off + mb;
     const bool valid = r < p.blk_n[blk];
     const long grow = (long)p.blk_row[blk] + r;
+    const float rs = p.row_scale ? p.row_scale[(size_t)mb * BM + r] : 1.0f;
     __nv_bfloat16* out = p.dHidden + (size_t)grow * p.dh_ld;
     for (int c0 = 0; c0 < BN; c0 += 32) {
       const int ncl = p.N - (n0 + c0);
@@ -251,10 +303,10 @@ __device__ __forceinline__ void epilogue_tile(const TcArgs& p, uint32_t tmem_acc
         for (int q = 0; q < 4; ++q) {
           if (q * 8 < ncl) {
             uint4 w;
-            w.x = pack_bf16x2(__uint_as_float(v[q * 8 + 0]), __uint_as_float(v[q * 8 + 1]));
-            w.y = pack_bf16x2(__uint_as_float(v[q * 8 + 2]), __uint_as_float(v[q * 8 + 3]));
-            w.z = pack_bf16x2(__uint_as_float(v[q * 8 + 4]), __uint_as_float(v[q * 8 + 5]));
-            w.w = pack_bf16x2(__uint_as_float(v[q * 8 + 6]), __uint_as_float(v[q * 8 + 7]));
+            w.x = pack_bf16x2(rs * __uint_as_float(v[q * 8 + 0]), rs * __uint_as_float(v[q * 8 + 1]));
+            w.y = pack_bf16x2(rs * __uint_as_float(v[q * 8 + 2]), rs * __uint_as_float(v[q * 8 + 3]));
+            w.z = pack_bf16x2(rs * __uint_as_float(v[q * 8 + 4]), rs * __uint_as_float(v[q * 8 + 5]));
+            w.w = pack_bf16x2(rs * __uint_as_float(v[q * 8 + 6]), rs * __uint_as_float(v[q * 8 + 7]));
             *reinterpret_cast<uint4*>(out + n0 + c0 + q * 8) = w;
           }
         }
@@ -341,7 +393,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x) {
         int mb, nt;
         tile_coords(tile, MB, NT, p.raster_band, mb, nt);
-        const int a_row = (EPI == TC_EPI_LSE || EPI == TC_EPI_DS) ? p.blk_row[p.blk_off + mb] : mb * BM;
+        const int a_row = (EPI == TC_EPI_LSE || EPI == TC_EPI_DS || EPI == TC_EPI_E) ? p.blk_row[p.blk_off + mb] : mb * BM;
         const int b_row = nt * BN;
         for (int kb = 0; kb < nkb; ++kb) {
           if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status))) break;
@@ -482,6 +534,7 @@ cudaError_t launch_tc_gemm(const TcGemm& g, cudaStream_t s) {
   a.ids = g.ids; a.lse = g.lse; a.g = g.g; a.partials = g.partials; a.tgt = g.tgt;
   a.dS = g.dS; a.ds_ld = g.ds_ld; a.dSt = g.dSt; a.dst_ld = g.dst_ld;
   a.dHidden = g.dHidden; a.dh_ld = g.dh_ld; a.dW = g.dW; a.dw_ld = g.dw_ld; a.status = g.status;
+  a.psum = g.psum; a.row_scale = g.row_scale;
   const int NT = cdiv(g.N, BN);
   const long max_tiles = (long)(g.epi == TC_EPI_DW ? g.m_blocks : g.blk_cap) * NT;
   const int grid = (int)(max_tiles < (long)tc_num_sms() ? (max_tiles > 0 ? max_tiles : 1) : tc_num_sms());
@@ -490,6 +543,7 @@ cudaError_t launch_tc_gemm(const TcGemm& g, cudaStream_t s) {
     case TC_EPI_DS: return launch_one<TC_EPI_DS>(tmA, tmB, a, grid, s);
     case TC_EPI_DH: return launch_one<TC_EPI_DH>(tmA, tmB, a, grid, s);
     case TC_EPI_DW: return launch_one<TC_EPI_DW>(tmA, tmB, a, grid, s);
+    case TC_EPI_E: return launch_one<TC_EPI_E>(tmA, tmB, a, grid, s);
   }
   return cudaErrorInvalidValue;
 }

@@ -110,13 +110,14 @@ def test_config2_backward_sampled_rows_full_dW(trl, cfg2_batch):
         assert rel_fro(dW_host[v], ref_dW[v]) <= 2 * TOL_GRAD
 
 
-def test_config2_whole_step_sampled_rows_and_invariants(trl, cfg2_batch):
+@pytest.mark.parametrize("fused", [False, True])
+def test_config2_whole_step_sampled_rows_and_invariants(trl, cfg2_batch, fused):
     """The whole path in the benchmark's launch configuration: log-probs, g and dHidden on
     sampled rows against a from-scratch oracle per row; integers over all tokens; invariants."""
     w, batch = cfg2_batch
     lens, bnd, ids = batch["lens"].cpu().numpy(), batch["bnd"].cpu().numpy(), batch["ids"].cpu().numpy()
     status = torch.zeros(1, dtype=torch.int32, device=DEV)
-    out = trl.hrd_pg_step(batch, w.P, w.G, w.T, status=status)
+    out = trl.hrd_pg_step(batch, w.P, w.G, w.T, status=status, fused=fused)
     torch.cuda.synchronize()
     trl.check_status(status)
     hrd_ref = orc.hrd_advantages(f64(batch["r_plan"]), f64(batch["r_code"]), lens, bnd, w.P, w.G, w.T)

@@ -19,7 +19,8 @@ def trl():
     return t
 
 
-def run_and_compare(trl, w, batch=None, explicit_old=False, alpha=0.1, eps=0.2, adv_mode=0):
+def run_and_compare(trl, w, batch=None, explicit_old=False, alpha=0.1, eps=0.2, adv_mode=0, fused=False,
+                    use_hint=True):
     dev = "cuda:0"
     batch = synth.make_batch(w, device=dev) if batch is None else batch
     oi = oracle_inputs(batch)
@@ -32,7 +33,8 @@ def run_and_compare(trl, w, batch=None, explicit_old=False, alpha=0.1, eps=0.2, 
     ref = orc.full_step(oi["hidden"], oi["W"], oi["hidden_old"], oi["W_old"], oi["ids"], oi["lens"], oi["bnd"],
                         oi["r_plan"], oi["r_code"], w.P, w.G, w.T, eps, eps, alpha, adv_mode, old_logp=old_logp_o)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
-    out = trl.hrd_pg_step(batch, w.P, w.G, w.T, eps, eps, alpha, adv_mode, old_logp=old_logp_g, status=status)
+    out = trl.hrd_pg_step(batch, w.P, w.G, w.T, eps, eps, alpha, adv_mode, old_logp=old_logp_g, status=status,
+                          fused=fused, use_hint=use_hint)
     torch.cuda.synchronize()
     trl.check_status(status)
     hrd = out["hrd"]
@@ -172,6 +174,50 @@ def test_host_argument_errors(trl):
     with pytest.raises(trl.TrlError, match="shape"):
         trl.trl_token_logprobs(batch["hidden"][:, :60].contiguous(), batch["W"][:, :60].contiguous(), batch["ids"],
                                batch["lens"], w.T)      # H % 8 != 0 in bf16
+
+
+@pytest.mark.parametrize("use_hint", [True, False])
+def test_fused_step_matches_oracle(trl, use_hint):
+    """trl_pg_step_fused (forward GEMM stores E = exp(z - c), no recompute) against the oracle,
+    with the old policy's lse as the shift and with no hint."""
+    w = synth.scaled(synth.CONFIGS[2], name="fused_ragged", P=2, G=4, T=300, H=320, V=1000)
+    run_and_compare(trl, w, fused=True, use_hint=use_hint)
+    run_and_compare(trl, w, fused=True, use_hint=use_hint, explicit_old=True, alpha=0.5, eps=0.1)
+    w = synth.scaled(synth.CONFIGS[2], name="fused_wide", P=3, G=6, T=384, H=512, V=3000, real_plan_reward=True,
+                     len_lo=0.1, degenerate_frac=0.34)
+    run_and_compare(trl, w, fused=True, use_hint=use_hint)
+    run_and_compare(trl, synth.CONFIGS[0], fused=True, use_hint=use_hint)          # fp32: three calls inside
+
+
+def test_fused_step_edge_cases(trl):
+    w = synth.scaled(synth.CONFIGS[2], name="fused_edge", P=2, G=4, T=160, H=128, V=512)
+    batch = synth.make_batch(w, device="cuda:0")
+    batch["lens"] = torch.tensor([0, 160, 1, 128, 129, 77, 0, 5], dtype=torch.int32).cuda()
+    batch["bnd"] = torch.tensor([0, 0, 1, 128, 64, 77, 0, 2], dtype=torch.int32).cuda()
+    run_and_compare(trl, w, batch=batch, fused=True)
+    batch["lens"], batch["bnd"] = torch.zeros(8, dtype=torch.int32).cuda(), torch.zeros(8, dtype=torch.int32).cuda()
+    out, _ = run_and_compare(trl, w, batch=batch, fused=True)
+    assert float(out["loss"]) == 0.0
+
+
+def test_fused_step_any_reasonable_hint_gives_same_result_and_bad_hint_is_flagged(trl):
+    w = synth.scaled(synth.CONFIGS[2], name="fused_hint", P=2, G=4, T=200, H=256, V=1536)
+    batch = synth.make_batch(w, device="cuda:0")
+    old_logp, old_lse = trl.trl_token_logprobs(batch["hidden_old"], batch["W_old"], batch["ids"], batch["lens"], w.T)
+    hrd = trl.trl_hrd_advantages(batch["r_plan"], batch["r_code"], batch["lens"], batch["bnd"], w.P, w.G, w.T)
+    args = (batch["hidden"], batch["W"], batch["ids"], batch["lens"], old_logp)
+    ref = trl.trl_pg_step_fused(*args, None, hrd["adv"], hrd["seg"], w.P, w.G, w.T)
+    shifted = old_lse + 10.0 * (torch.rand_like(old_lse) - 0.5)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda:0")
+    out = trl.trl_pg_step_fused(*args, shifted, hrd["adv"], hrd["seg"], w.P, w.G, w.T, status=status)
+    torch.cuda.synchronize()
+    trl.check_status(status)
+    assert (out["logp"] - ref["logp"]).abs().max() <= 1e-4
+    assert abs(float(out["loss"]) - float(ref["loss"])) <= 1e-4 * abs(float(ref["loss"]))
+    assert rel_fro(f64(out["dW"]), f64(ref["dW"])) <= 1e-2 and rel_fro(f64(out["dHidden"]), f64(ref["dHidden"])) <= 1e-2
+    trl.trl_pg_step_fused(*args, old_lse - 500.0, hrd["adv"], hrd["seg"], w.P, w.G, w.T, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) & (1 << 9)
 
 
 def test_minimum_workspace_gives_same_backward(trl):
