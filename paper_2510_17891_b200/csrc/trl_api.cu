@@ -44,9 +44,9 @@ size_t fwd_bytes_bf16(int B, int T, int V) {
 size_t fwd_bytes_f32(int B, int T, int H, int V, int R) {
   return row_blocks_bytes(B, T) + align_up((size_t)R * H * 4, 256) + align_up((size_t)R * V * 4, 256);
 }
-size_t bwd_fixed_bf16(int B, int T, int H, int V) { return row_blocks_bytes(B, T) + align_up((size_t)H * V * 2, 256); }
+size_t bwd_fixed_bf16(int B, int T, int H, int V) { (void)H; (void)V; return row_blocks_bytes(B, T); }
 size_t bwd_per_rows_bf16(int H, int V, int R) {
-  return align_up((size_t)H * R * 2, 256) + 2 * align_up((size_t)R * V * 2, 256);
+  return align_up((size_t)H * R * 2, 256) + align_up((size_t)R * V * 2, 256);   // gathered hidden rows + dS / E
 }
 size_t bwd_bytes_f32(int B, int T, int H, int V, int R) {
   return row_blocks_bytes(B, T) + 2 * align_up((size_t)R * H * 4, 256) + align_up((size_t)R * V * 4, 256);
@@ -236,14 +236,11 @@ int trl_pg_loss_bwd(const void* hidden, const void* W, const int32_t* ids, const
     const int R = fit_rows(avail, cap_rows < kRecommendedChunkRowsBf16 ? cap_rows : kRecommendedChunkRowsBf16,
                            [&](int r) { return bwd_per_rows_bf16(H, V, r); });
     if (R < kRowBlock) return TRL_ERR_WORKSPACE_TOO_SMALL;
-    __nv_bfloat16* Wt = cv.take<__nv_bfloat16>((size_t)H * V);
-    __nv_bfloat16* Xt = cv.take<__nv_bfloat16>((size_t)H * R);
+    __nv_bfloat16* Xs = cv.take<__nv_bfloat16>((size_t)H * R);
     __nv_bfloat16* dS = cv.take<__nv_bfloat16>((size_t)R * V);
-    __nv_bfloat16* dSt = cv.take<__nv_bfloat16>((size_t)V * R);
-    launch_transpose_bf16((const __nv_bfloat16*)W, Wt, V, H, s);
     const int CB = R / kRowBlock;
     for (int blk_off = 0; blk_off < rb.cap; blk_off += CB) {
-      launch_gather_transpose_bf16((const __nv_bfloat16*)hidden, Xt, H, R, rb, blk_off, nullptr, s);
+      launch_gather_rows_bf16((const __nv_bfloat16*)hidden, Xs, H, R, rb, blk_off, nullptr, s);
       TcGemm a;
       memset(&a, 0, sizeof(a));
       a.rb = rb; a.blk_off = blk_off; a.blk_cap = CB; a.status = status_dev;
@@ -251,18 +248,18 @@ int trl_pg_loss_bwd(const void* hidden, const void* W, const int32_t* ids, const
       TcGemm ds = a;
       ds.epi = TC_EPI_DS; ds.raster_band = kRasterBandFwd;
       ds.A = hidden; ds.a_rows = (long)N; ds.a_ld = H; ds.B = W; ds.b_rows = V; ds.b_ld = H; ds.K = H; ds.N = V;
-      ds.ids = ids; ds.lse = lse; ds.g = g; ds.dS = dS; ds.ds_ld = V; ds.dSt = dSt; ds.dst_ld = R;
+      ds.ids = ids; ds.lse = lse; ds.g = g; ds.dS = dS; ds.ds_ld = V;
       TRL_CUDA_OK(launch_tc_gemm(ds, s));
-      // dHidden rows of the chunk = dS W
+      // dHidden rows of the chunk = dS W   (W read as an N-contiguous operand)
       TcGemm dh = a;
       dh.epi = TC_EPI_DH; dh.raster_band = kRasterBandBwd;
-      dh.A = dS; dh.a_rows = R; dh.a_ld = V; dh.B = Wt; dh.b_rows = H; dh.b_ld = V; dh.K = V; dh.N = H;
+      dh.A = dS; dh.a_rows = R; dh.a_ld = V; dh.B = W; dh.b_rows = H; dh.b_ld = H; dh.K = V; dh.N = H;
       dh.dHidden = (__nv_bfloat16*)dHidden; dh.dh_ld = H;
       TRL_CUDA_OK(launch_tc_gemm(dh, s));
-      // dW += dS^T hidden
+      // dW += dS^T hidden   (both operands M/N-contiguous: dS [R,V] and the gathered rows [R,H])
       TcGemm dw = a;
       dw.epi = TC_EPI_DW; dw.raster_band = kRasterBandBwd;
-      dw.A = dSt; dw.a_rows = V; dw.a_ld = R; dw.B = Xt; dw.b_rows = H; dw.b_ld = R; dw.K = R; dw.N = H;
+      dw.A = dS; dw.a_rows = V; dw.a_ld = V; dw.B = Xs; dw.b_rows = H; dw.b_ld = H; dw.K = R; dw.N = H;
       dw.m_blocks = cdiv(V, kRowBlock); dw.dW = dW; dw.dw_ld = H; dw.V = V;
       TRL_CUDA_OK(launch_tc_gemm(dw, s));
     }
@@ -331,11 +328,9 @@ int trl_pg_step_fused(const void* hidden, const void* W, const int32_t* ids, con
 
   Carver cv(workspace);
   RowBlocks rb = carve_row_blocks(cv.take<char>(row_blocks_bytes(B, T)), B, T);
-  __nv_bfloat16* Wt = cv.take<__nv_bfloat16>((size_t)H * V);
   float* loss_partials = cv.take<float>((size_t)B * pg_loss_tiles(T) * 4);
-  __nv_bfloat16* Xt = cv.take<__nv_bfloat16>((size_t)H * R);
+  __nv_bfloat16* Xs = cv.take<__nv_bfloat16>((size_t)H * R);
   __nv_bfloat16* E = cv.take<__nv_bfloat16>((size_t)R * V);
-  __nv_bfloat16* Et = cv.take<__nv_bfloat16>((size_t)V * R);
   float* psum = cv.take<float>((size_t)nt * R);
   float* tgt = cv.take<float>(R);
   float* neg_alpha = cv.take<float>(R);
@@ -362,7 +357,6 @@ int trl_pg_step_fused(const void* hidden, const void* W, const int32_t* ids, con
     hint = lse;
   }
 
-  launch_transpose_bf16((const __nv_bfloat16*)W, Wt, V, H, s);
   const int CB = R / kRowBlock;
   for (int blk_off = 0; blk_off < rb.cap; blk_off += CB) {
     TcGemm a = base;
@@ -371,22 +365,22 @@ int trl_pg_step_fused(const void* hidden, const void* W, const int32_t* ids, con
     TcGemm e = a;
     e.epi = TC_EPI_E; e.raster_band = kRasterBandFwd;
     e.A = hidden; e.a_rows = (long)N; e.a_ld = H; e.B = W; e.b_rows = V; e.b_ld = H; e.K = H; e.N = V;
-    e.ids = ids; e.lse = hint; e.dS = E; e.ds_ld = V; e.dSt = Et; e.dst_ld = R; e.psum = psum; e.tgt = tgt; e.rows_cap = R;
+    e.ids = ids; e.lse = hint; e.dS = E; e.ds_ld = V; e.psum = psum; e.tgt = tgt; e.rows_cap = R;
     TRL_CUDA_OK(launch_tc_gemm(e, s));
     FusedMergeArgs m{psum, tgt, nt, R, rb, blk_off, ids, len, hint, old_logp, adv, seg, P, G, T, V, cfg,
-                     logp, lse, g, neg_alpha, E, Et, status_dev};
+                     logp, lse, g, neg_alpha, E, status_dev};
     launch_fused_merge(m, s);
-    launch_gather_transpose_bf16((const __nv_bfloat16*)hidden, Xt, H, R, rb, blk_off, neg_alpha, s);
+    launch_gather_rows_bf16((const __nv_bfloat16*)hidden, Xs, H, R, rb, blk_off, neg_alpha, s);
     // dHidden rows = neg_alpha * (E' W)
     TcGemm dh = a;
     dh.epi = TC_EPI_DH; dh.raster_band = kRasterBandBwd;
-    dh.A = E; dh.a_rows = R; dh.a_ld = V; dh.B = Wt; dh.b_rows = H; dh.b_ld = V; dh.K = V; dh.N = H;
+    dh.A = E; dh.a_rows = R; dh.a_ld = V; dh.B = W; dh.b_rows = H; dh.b_ld = H; dh.K = V; dh.N = H;
     dh.dHidden = (__nv_bfloat16*)dHidden; dh.dh_ld = H; dh.row_scale = neg_alpha;
     TRL_CUDA_OK(launch_tc_gemm(dh, s));
     // dW += E'^T (neg_alpha * hidden)
     TcGemm dw = a;
     dw.epi = TC_EPI_DW; dw.raster_band = kRasterBandBwd;
-    dw.A = Et; dw.a_rows = V; dw.a_ld = R; dw.B = Xt; dw.b_rows = H; dw.b_ld = R; dw.K = R; dw.N = H;
+    dw.A = E; dw.a_rows = V; dw.a_ld = V; dw.B = Xs; dw.b_rows = H; dw.b_ld = H; dw.K = R; dw.N = H;
     dw.m_blocks = cdiv(V, kRowBlock); dw.dW = dW; dw.dw_ld = H; dw.V = V;
     TRL_CUDA_OK(launch_tc_gemm(dw, s));
   }

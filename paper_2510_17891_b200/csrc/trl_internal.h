@@ -44,11 +44,10 @@ void launch_pg_loss(const float* logp, const float* old_logp, const float* adv, 
 void launch_merge_lse(const float2* partials, const float* tgt, int n_tiles, int rows_cap, RowBlocks rb,
                       const int32_t* ids, const int32_t* len, int B, int T, int V, float* logp, float* lse,
                       int32_t* status, cudaStream_t s);
-void launch_transpose_bf16(const __nv_bfloat16* in, __nv_bfloat16* out, int rows, int cols, cudaStream_t s);
-// Xt[h, r] = hidden[row(blk_off*128 + r), h] for the live rows of a chunk, 0 elsewhere
-// (times col_scale[r] when given)
-void launch_gather_transpose_bf16(const __nv_bfloat16* hidden, __nv_bfloat16* Xt, int H, int R, RowBlocks rb,
-                                  int blk_off, const float* col_scale, cudaStream_t s);
+// Xs[r, :] = hidden[row(blk_off*128 + r), :] for the live rows of a chunk (times
+// row_scale[r] when given), 0 elsewhere
+void launch_gather_rows_bf16(const __nv_bfloat16* hidden, __nv_bfloat16* Xs, int H, int R, RowBlocks rb,
+                             int blk_off, const float* row_scale, cudaStream_t s);
 // Chunk-local finish of the fused step: lse = c + log(sum_k psum), logp, g = d loss/d logp,
 // the per-row factor -g exp(c - lse) for the gradient GEMMs, and the one-hot fix of E / E^T.
 struct FusedMergeArgs {
@@ -56,7 +55,7 @@ struct FusedMergeArgs {
   const int32_t* ids; const int32_t* len; const float* hint; const float* old_logp; const float* adv;
   const uint8_t* seg; int P, G, T, V; trl_pg_config cfg;
   float* logp; float* lse; float* g; float* neg_alpha;
-  __nv_bfloat16* E; __nv_bfloat16* Et;
+  __nv_bfloat16* E;
   int32_t* status;
 };
 void launch_fused_merge(const FusedMergeArgs& a, cudaStream_t s);
@@ -87,8 +86,10 @@ void launch_simt_gemm(const SimtGemm& p, cudaStream_t s);
 enum TcEpilogue { TC_EPI_LSE = 0, TC_EPI_DS = 1, TC_EPI_DH = 2, TC_EPI_DW = 3, TC_EPI_E = 4 };
 struct TcGemm {
   int epi;
-  // operands: A [a_rows, K] and B [b_rows, K], both bf16 row-major with K contiguous
-  const void* A; long a_rows; long a_ld;     // a_ld = row pitch in elements
+  // operands, bf16.  a_rows / b_rows = extent of the M / N dimension, K = extent of the
+  // contraction.  K-major operand (forward; A of DH): stored [rows, K], pitch ld.  MN-major
+  // operand (B of DH; A and B of DW): stored [K, rows], pitch ld.
+  const void* A; long a_rows; long a_ld;
   const void* B; long b_rows; long b_ld;
   int K;                                     // host K extent (TC_EPI_DW: K = 128 * live blocks of the chunk)
   int N;                                     // GEMM N extent = b_rows that are meaningful
@@ -98,7 +99,7 @@ struct TcGemm {
   // epilogue arguments
   const int32_t* ids; const float* lse; const float* g;
   float2* partials; float* tgt; int rows_cap;          // LSE
-  __nv_bfloat16* dS; long ds_ld; __nv_bfloat16* dSt; long dst_ld;   // DS
+  __nv_bfloat16* dS; long ds_ld;                       // DS, E
   __nv_bfloat16* dHidden; long dh_ld;                  // DH
   float* dW; long dw_ld; int V;                        // DW
   float* psum;                                         // E: row sums per vocabulary tile [n_tiles, rows_cap]

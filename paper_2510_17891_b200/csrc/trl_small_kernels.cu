@@ -311,60 +311,41 @@ void launch_merge_lse(const float2* partials, const float* tgt, int n_tiles, int
 }
 
 // ------------------------------------------------------------------------------------
-// bf16 transposes (64x64 tiles through shared memory)
+// Gathered (and optionally scaled) hidden rows of a chunk: the B operand of dW = dS^T hidden.
+// One CTA per scratch row; 16-byte loads and stores.
 // ------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) transpose_bf16_kernel(const __nv_bfloat16* __restrict__ in,
-                                                             __nv_bfloat16* __restrict__ out, int rows, int cols) {
-  __shared__ __nv_bfloat16 tile[64][66];
-  const int r0 = blockIdx.y * 64, c0 = blockIdx.x * 64;
-  const int tx = threadIdx.x & 63, ty = threadIdx.x >> 6;
-  for (int i = ty; i < 64; i += 4) {
-    const int r = r0 + i, c = c0 + tx;
-    tile[i][tx] = (r < rows && c < cols) ? in[(size_t)r * cols + c] : __float2bfloat16(0.f);
+__global__ void __launch_bounds__(128) gather_rows_bf16_kernel(const __nv_bfloat16* __restrict__ hidden,
+                                                               __nv_bfloat16* __restrict__ Xs, int H, int R,
+                                                               RowBlocks rb, int blk_off,
+                                                               const float* __restrict__ row_scale) {
+  const int r = blockIdx.x;
+  const int blk = blk_off + r / kRowBlock;
+  const int lr = r % kRowBlock;
+  const bool live = blk < rb.nblk[0] && lr < rb.blk_n[blk];
+  uint4* dst = reinterpret_cast<uint4*>(Xs + (size_t)r * H);
+  if (!live) {
+    for (int i = threadIdx.x; i < H / 8; i += 128) dst[i] = make_uint4(0, 0, 0, 0);
+    return;
   }
-  __syncthreads();
-  for (int i = ty; i < 64; i += 4) {
-    const int c = c0 + i, r = r0 + tx;
-    if (c < cols && r < rows) out[(size_t)c * rows + r] = tile[tx][i];
-  }
-}
-
-void launch_transpose_bf16(const __nv_bfloat16* in, __nv_bfloat16* out, int rows, int cols, cudaStream_t s) {
-  dim3 grid(cdiv(cols, 64), cdiv(rows, 64));
-  transpose_bf16_kernel<<<grid, 256, 0, s>>>(in, out, rows, cols);
-  note_launch();
-}
-
-// Xt [H, R]: column r is hidden row (block blk_off + r/128, lane r%128) or 0 if not live.
-__global__ void __launch_bounds__(256) gather_transpose_bf16_kernel(const __nv_bfloat16* __restrict__ hidden,
-                                                                    __nv_bfloat16* __restrict__ Xt, int H, int R,
-                                                                    RowBlocks rb, int blk_off,
-                                                                    const float* __restrict__ col_scale) {
-  __shared__ __nv_bfloat16 tile[64][66];
-  const int r0 = blockIdx.y * 64, h0 = blockIdx.x * 64;     // r0: scratch row, 64 | 128 so one block per tile
-  const int blk = blk_off + r0 / kRowBlock;
-  const int live = blk < rb.nblk[0];
-  const int tx = threadIdx.x & 63, ty = threadIdx.x >> 6;
-  const long grow0 = live ? (long)rb.blk_row[blk] : 0;
-  const int nvalid = live ? rb.blk_n[blk] : 0;
-  for (int i = ty; i < 64; i += 4) {
-    const int lr = (r0 % kRowBlock) + i;
-    const int h = h0 + tx;
-    __nv_bfloat16 x = (lr < nvalid && h < H) ? hidden[(size_t)(grow0 + lr) * H + h] : __float2bfloat16(0.f);
-    if (col_scale && lr < nvalid) x = __float2bfloat16_rn(__bfloat162float(x) * col_scale[r0 + i]);
-    tile[i][tx] = x;
-  }
-  __syncthreads();
-  for (int i = ty; i < 64; i += 4) {
-    const int h = h0 + i, r = r0 + tx;
-    if (h < H && r < R) Xt[(size_t)h * R + r] = tile[tx][i];
+  const uint4* src = reinterpret_cast<const uint4*>(hidden + ((size_t)rb.blk_row[blk] + lr) * H);
+  const float sc = row_scale ? row_scale[r] : 1.0f;
+  for (int i = threadIdx.x; i < H / 8; i += 128) {
+    uint4 x = src[i];
+    if (row_scale) {
+      __nv_bfloat162* h2 = reinterpret_cast<__nv_bfloat162*>(&x);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        float2 f = __bfloat1622float2(h2[q]);
+        h2[q] = __floats2bfloat162_rn(f.x * sc, f.y * sc);
+      }
+    }
+    dst[i] = x;
   }
 }
 
-void launch_gather_transpose_bf16(const __nv_bfloat16* hidden, __nv_bfloat16* Xt, int H, int R, RowBlocks rb,
-                                  int blk_off, const float* col_scale, cudaStream_t s) {
-  dim3 grid(cdiv(H, 64), cdiv(R, 64));
-  gather_transpose_bf16_kernel<<<grid, 256, 0, s>>>(hidden, Xt, H, R, rb, blk_off, col_scale);
+void launch_gather_rows_bf16(const __nv_bfloat16* hidden, __nv_bfloat16* Xs, int H, int R, RowBlocks rb, int blk_off,
+                             const float* row_scale, cudaStream_t s) {
+  gather_rows_bf16_kernel<<<R, 128, 0, s>>>(hidden, Xs, H, R, rb, blk_off, row_scale);
   note_launch();
 }
 
@@ -373,7 +354,7 @@ void launch_gather_transpose_bf16(const __nv_bfloat16* hidden, __nv_bfloat16* Xt
 //   lse = c + log sum_v E,  logp = z[id] - lse,  g = d loss / d logp (same formula as
 //   pg_loss_stage1_kernel),  dS = g onehot - g exp(c - lse) E = neg_alpha (E - exp(lse - c) onehot),
 // so the kernel stores neg_alpha = -g exp(c - lse) and subtracts exp(lse - c) from the
-// sampled token's entry of E and E^T.
+// sampled token's entry of E.
 // ------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(128) fused_merge_kernel(FusedMergeArgs a) {
   const int r = blockIdx.x * 128 + threadIdx.x;
@@ -409,9 +390,7 @@ __global__ void __launch_bounds__(128) fused_merge_kernel(FusedMergeArgs a) {
   if (gn != 0.f) {
     const float beta = expf(lse - c);
     __nv_bfloat16* e = a.E + (size_t)r * a.V + id;
-    const __nv_bfloat16 fixed = __float2bfloat16_rn(__bfloat162float(*e) - beta);
-    *e = fixed;
-    a.Et[(size_t)id * a.R + r] = fixed;
+    *e = __float2bfloat16_rn(__bfloat162float(*e) - beta);
   }
 }
 

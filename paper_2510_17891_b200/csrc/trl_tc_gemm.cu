@@ -1,15 +1,17 @@
 // tcgen05 / TMEM bf16 GEMM family for sm_100a.
 //
-// One persistent, warp-specialised kernel computes C[m,n] = sum_k A[m,k] B[n,k] (both
-// operands K-contiguous bf16, fp32 accumulation in tensor memory) on 128x256 tiles and
-// applies one of four epilogues straight from TMEM:
+// One persistent, warp-specialised kernel computes C[m,n] = sum_k A[m,k] B[n,k] (bf16
+// operands, fp32 accumulation in tensor memory) on 128x256 tiles.  Each operand is read in
+// the layout it already has in memory: K-contiguous ("K-major": hidden and W in the forward,
+// dS / E in dHidden = dS W) or M/N-contiguous ("MN-major": W in dHidden = dS W, dS / E and the
+// gathered hidden rows in dW = dS^T hidden), so no operand is ever transposed in memory.
+// One of five epilogues is applied straight from TMEM:
 //   LSE : per-row (max, sum-exp) of the tile's logits + pick-up of the sampled token's
 //         logit                                       (token scoring, Section 2.3 ratio s)
-//   DS  : dS = g (onehot - exp(z - lse)) as bf16, written row-major and transposed
+//   DS  : dS = g (onehot - exp(z - lse)) as bf16
 //   DH  : dHidden rows (bf16), scattered to the caller's row positions
 //   DW  : dW += tile (fp32 read-modify-write)
-//   E   : E = exp(z - c) for a per-row shift c (a stale log-partition), as bf16 row-major
-//         and transposed, plus the row sums of E and the sampled token's logit.  The softmax
+//   E   : E = exp(z - c) for a per-row shift c (a stale log-partition), as bf16, plus the row sums of E and the sampled token's logit.  The softmax
 //         is p = E exp(c - lse), a per-row factor the gradient GEMMs fold into their other
 //         operand / their epilogue, so the forward GEMM is not repeated in the backward.
 //
@@ -40,7 +42,7 @@ struct TcArgs {
   const int* nblk; const int* blk_row; const int* blk_n;
   const int32_t* ids; const float* lse; const float* g;
   float2* partials; float* tgt;
-  __nv_bfloat16* dS; long ds_ld; __nv_bfloat16* dSt; long dst_ld;
+  __nv_bfloat16* dS; long ds_ld;
   __nv_bfloat16* dHidden; long dh_ld;
   float* dW; long dw_ld;
   float* psum; const float* row_scale;
@@ -138,10 +140,27 @@ __device__ __forceinline__ uint64_t make_kmajor_sw128_desc(uint32_t smem_addr) {
   d |= (uint64_t)2 << 61;
   return d;
 }
-// Instruction descriptor, kind::f16: D = fp32, A = B = bf16, both K-major, M x N tile.
-__host__ __device__ constexpr uint32_t make_idesc_bf16(int M, int N) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+// MN-major operand, 128-byte swizzle.  The tile is stored as groups of 64 M/N-elements:
+// inside a group every k-row is 128 contiguous bytes, 8 k-rows form a 1024 B swizzle atom
+// (stride byte offset = distance between 8-row atoms along K = 1024 B), and groups follow
+// each other every 64 k-rows x 128 B = 8192 B (leading byte offset).
+__device__ __forceinline__ uint64_t make_mnmajor_sw128_desc(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr >> 4) & 0x3FFF);
+  d |= (uint64_t)(8192 >> 4) << 16;
+  d |= (uint64_t)(1024 >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
 }
+// Instruction descriptor, kind::f16: D = fp32, A = B = bf16, M x N tile; bit 15 / 16 select
+// an MN-major A / B operand.
+__host__ __device__ constexpr uint32_t make_idesc_bf16(int M, int N, bool a_mn, bool b_mn) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
+         ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+__host__ __device__ constexpr bool a_is_mn(int epi) { return epi == TC_EPI_DW; }
+__host__ __device__ constexpr bool b_is_mn(int epi) { return epi == TC_EPI_DW || epi == TC_EPI_DH; }
 
 __device__ __forceinline__ void tile_coords(int tile, int MB, int NT, int band_rows, int& mb, int& nt) {
   const int per_band = band_rows * NT;
@@ -236,10 +255,6 @@ __device__ __forceinline__ void epilogue_tile(const TcArgs& p, uint32_t tmem_acc
           *reinterpret_cast<uint4*>(ds_row + n0 + c0 + q * 8) = w;
         }
       }
-      __nv_bfloat16* dst_col = p.dSt + (size_t)(n0 + c0) * p.dst_ld + srow;
-#pragma unroll
-      for (int j = 0; j < 32; ++j)
-        if (j < ncl) dst_col[(size_t)j * p.dst_ld] = __float2bfloat16_rn(d[j]);
     }
   } else if constexpr (EPI == TC_EPI_E) {
     const int blk = p.blk_off + mb;
@@ -280,10 +295,6 @@ __device__ __forceinline__ void epilogue_tile(const TcArgs& p, uint32_t tmem_acc
           *reinterpret_cast<uint4*>(e_row + n0 + c0 + q * 8) = w;
         }
       }
-      __nv_bfloat16* et_col = p.dSt + (size_t)(n0 + c0) * p.dst_ld + srow;
-#pragma unroll
-      for (int j = 0; j < 32; ++j)
-        if (j < ncl) et_col[(size_t)j * p.dst_ld] = __float2bfloat16_rn(d[j]);
     }
     p.psum[(size_t)nt * p.rows_cap + srow] = sum;
     if (has) p.tgt[srow] = tg;
@@ -399,8 +410,19 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status))) break;
           mbar_expect_tx(full_bar(stage), STAGE_BYTES);
           const uint32_t sa = smem_base + stage * STAGE_BYTES;
-          tma_load_2d(sa, &tmA, kb * BK, a_row, full_bar(stage));
-          tma_load_2d(sa + A_BYTES, &tmB, kb * BK, b_row, full_bar(stage));
+          if constexpr (a_is_mn(EPI)) {       // two 64(M) x 64(K) boxes
+            tma_load_2d(sa, &tmA, a_row, kb * BK, full_bar(stage));
+            tma_load_2d(sa + 8192, &tmA, a_row + 64, kb * BK, full_bar(stage));
+          } else {
+            tma_load_2d(sa, &tmA, kb * BK, a_row, full_bar(stage));
+          }
+          if constexpr (b_is_mn(EPI)) {       // four 64(N) x 64(K) boxes
+#pragma unroll
+            for (int j = 0; j < BN / 64; ++j)
+              tma_load_2d(sa + A_BYTES + j * 8192, &tmB, b_row + 64 * j, kb * BK, full_bar(stage));
+          } else {
+            tma_load_2d(sa + A_BYTES, &tmB, kb * BK, b_row, full_bar(stage));
+          }
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
       }
@@ -412,7 +434,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      constexpr uint32_t idesc = make_idesc_bf16(BM, BN);
+      constexpr uint32_t idesc = make_idesc_bf16(BM, BN, a_is_mn(EPI), b_is_mn(EPI));
       int stage = 0; uint32_t phase = 0;
       int acc = 0; uint32_t acc_phase = 0;
       bool ok = true;
@@ -424,13 +446,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           if (!(ok = mbar_wait(full_bar(stage), phase, abort_flag, p.status))) break;
           tc_fence_after();
           const uint32_t sa = smem_base + stage * STAGE_BYTES;
-          const uint64_t da = make_kmajor_sw128_desc(sa);
-          const uint64_t db = make_kmajor_sw128_desc(sa + A_BYTES);
+          const uint64_t da = a_is_mn(EPI) ? make_mnmajor_sw128_desc(sa) : make_kmajor_sw128_desc(sa);
+          const uint64_t db = b_is_mn(EPI) ? make_mnmajor_sw128_desc(sa + A_BYTES) : make_kmajor_sw128_desc(sa + A_BYTES);
+          // one MMA consumes 16 k.  K-major: 32 B further along the 128 B swizzle row (+2 in the
+          // >>4 address field).  MN-major: two 8-row atoms of 1024 B further (+128).
+          constexpr uint64_t ka = a_is_mn(EPI) ? 128 : 2, kbs = b_is_mn(EPI) ? 128 : 2;
 #pragma unroll
-          for (int k = 0; k < BK / UMMA_K; ++k) {
-            // advance 32 B (16 bf16) along K inside the 128 B swizzle row: +2 in the >>4 address field
-            tc_mma_bf16(d_tmem, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (uint32_t)((kb | k) != 0));
-          }
+          for (int k = 0; k < BK / UMMA_K; ++k)
+            tc_mma_bf16(d_tmem, da + ka * k, db + kbs * k, idesc, (uint32_t)((kb | k) != 0));
           tc_commit(empty_bar(stage));
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
@@ -485,12 +508,13 @@ EncodeTiledFn get_encode_fn() {
 }
 
 // 2-D bf16 tensor [rows, K] with row pitch `ld` elements; box = [box_rows, 64] elements, 128 B swizzle.
-bool make_tmap(CUtensorMap* tm, const void* base, long rows, long K, long ld, int box_rows) {
+// (MN-major operand: stored [K, mn] with mn contiguous; box = 64 (mn) x 64 (k).)
+bool make_tmap(CUtensorMap* tm, const void* base, long rows, long K, long ld, int box_rows, bool mn_major) {
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) return false;
-  cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+  cuuint64_t dims[2] = {(cuuint64_t)(mn_major ? rows : K), (cuuint64_t)(mn_major ? K : rows)};
   cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
-  cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
+  cuuint32_t box[2] = {(cuuint32_t)64, (cuuint32_t)(mn_major ? BK : box_rows)};
   cuuint32_t estr[2] = {1, 1};
   CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -525,14 +549,14 @@ int tc_num_sms() {
 
 cudaError_t launch_tc_gemm(const TcGemm& g, cudaStream_t s) {
   CUtensorMap tmA, tmB;
-  if (!make_tmap(&tmA, g.A, g.a_rows, g.K, g.a_ld, BM)) return cudaErrorInvalidValue;
-  if (!make_tmap(&tmB, g.B, g.b_rows, g.K, g.b_ld, BN)) return cudaErrorInvalidValue;
+  if (!make_tmap(&tmA, g.A, g.a_rows, g.K, g.a_ld, BM, a_is_mn(g.epi))) return cudaErrorInvalidValue;
+  if (!make_tmap(&tmB, g.B, g.b_rows, g.K, g.b_ld, BN, b_is_mn(g.epi))) return cudaErrorInvalidValue;
   TcArgs a;
   a.N = g.N; a.K = g.K; a.m_blocks_fixed = g.m_blocks; a.blk_off = g.blk_off; a.blk_cap = g.blk_cap;
   a.raster_band = g.raster_band > 0 ? g.raster_band : 16; a.rows_cap = g.rows_cap; a.V = g.V;
   a.nblk = g.rb.nblk; a.blk_row = g.rb.blk_row; a.blk_n = g.rb.blk_n;
   a.ids = g.ids; a.lse = g.lse; a.g = g.g; a.partials = g.partials; a.tgt = g.tgt;
-  a.dS = g.dS; a.ds_ld = g.ds_ld; a.dSt = g.dSt; a.dst_ld = g.dst_ld;
+  a.dS = g.dS; a.ds_ld = g.ds_ld;
   a.dHidden = g.dHidden; a.dh_ld = g.dh_ld; a.dW = g.dW; a.dw_ld = g.dw_ld; a.status = g.status;
   a.psum = g.psum; a.row_scale = g.row_scale;
   const int NT = cdiv(g.N, BN);
