@@ -10,7 +10,7 @@
 //         logit                                       (token scoring, Section 2.3 ratio s)
 //   DS  : dS = g (onehot - exp(z - lse)) as bf16
 //   DH  : dHidden rows (bf16), scattered to the caller's row positions
-//   DW  : dW += tile (fp32 read-modify-write)
+//   DW  : dW += tile (fp32, TMA reduce-add from shared memory)
 //   E   : E = exp(z - c) for a per-row shift c (a stale log-partition), as bf16, plus the row sums of E and the sampled token's logit.  The softmax
 //         is p = E exp(c - lse), a per-row factor the gradient GEMMs fold into their other
 //         operand / their epilogue, so the forward GEMM is not repeated in the backward.
@@ -19,6 +19,8 @@
 // and TMEM owner, warps 2..5 = epilogue (one TMEM lane quadrant each).  Shared-memory
 // stages are guarded by full/empty mbarriers; the 512 TMEM columns hold two 128x256 fp32
 // accumulators so the epilogue of tile i overlaps the mainloop of tile i+1.
+// The dS / E / dW epilogues stage 32-row x 128-byte units in swizzled shared memory and hand
+// them to the TMA (bulk tensor store / reduce-add), so global memory sees whole 128 B lines.
 // Every wait is bounded: on expiry the CTA raises TRL_ERR_TIMEOUT in the status word,
 // all roles leave their loops, TMEM is freed and the kernel returns.
 #include <cuda.h>
@@ -31,7 +33,8 @@ namespace {
 
 constexpr int BM = 128, BN = 256, BK = 64, UMMA_K = 16, STAGES = 4;
 constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int OUT_STAGE_BYTES = 4 * 2 * 4096;   // 4 epilogue warps x 2 buffers x (32 rows x 128 B)
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + OUT_STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr int NUM_THREADS = 192;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr float LOG2E = 1.4426950408889634f, LN2 = 0.6931471805599453f;
@@ -175,10 +178,51 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&h);
 }
 
+// Per-warp staged output: each lane owns one 128-byte row of a 32-row unit.  Rows are
+// written with the 128-byte swizzle (16-byte chunk index XOR row%8) the tensor map expects,
+// then one lane issues the bulk tensor store (or fp32 reduce-add); two buffers alternate.
+struct WarpOut {
+  uint32_t smem;            // this warp's two 4 KB buffers, 1024-byte aligned
+  const CUtensorMap* tm;
+  int lane;
+  int n;
+  template <bool REDUCE>
+  __device__ __forceinline__ void put(const uint4 (&w)[8], int x, int y) {
+    const uint32_t buf = smem + (uint32_t)(n & 1) * 4096u;
+    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+    __syncwarp();
+    const uint32_t row = buf + (uint32_t)lane * 128u;
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+      asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row + (uint32_t)((j ^ (lane & 7)) << 4)), "r"(w[j].x),
+                   "r"(w[j].y), "r"(w[j].z), "r"(w[j].w)
+                   : "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    __syncwarp();
+    if (lane == 0) {
+      if constexpr (REDUCE)
+        asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.bulk_group [%0, {%2, %3}], [%1];" ::"l"(tm),
+                     "r"(buf), "r"(x), "r"(y)
+                     : "memory");
+      else
+        asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(tm), "r"(buf),
+                     "r"(x), "r"(y)
+                     : "memory");
+      asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+    }
+    ++n;
+  }
+  __device__ __forceinline__ void drain() {
+    if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    __syncwarp();
+  }
+};
+
 // ---------------------------------------------------------------- epilogues
 // Each epilogue thread owns one accumulator row (TMEM lane) of the 128x256 tile.
 template <int EPI>
-__device__ __forceinline__ void epilogue_tile(const TcArgs& p, uint32_t tmem_acc, int quad, int lane, int mb, int nt) {
+__device__ __forceinline__ void epilogue_tile(const TcArgs& p, uint32_t tmem_acc, int quad, int lane, int mb, int nt,
+                                              WarpOut& wo) {
   const int r = quad * 32 + lane;           // row within the tile
   const int n0 = nt * BN;
   const uint32_t taddr = tmem_acc + ((uint32_t)(quad * 32) << 16);
@@ -229,32 +273,27 @@ __device__ __forceinline__ void epilogue_tile(const TcArgs& p, uint32_t tmem_acc
     const int id = valid ? p.ids[grow] : -1;
     const float gg = valid ? p.g[grow] : 0.f;
     const float L2 = valid ? p.lse[grow] * LOG2E : 0.f;
-    const size_t srow = (size_t)mb * BM + r;
-    __nv_bfloat16* ds_row = p.dS + srow * p.ds_ld;
-    for (int c0 = 0; c0 < BN; c0 += 32) {
-      const int ncl = p.N - (n0 + c0);
-      if (ncl <= 0) break;
-      tc_ld32(taddr + c0, v);
-      tc_wait_ld();
-      float d[32];
-      const int lc = id - (n0 + c0);
+    const bool live = valid && gg != 0.f;
+    for (int c0 = 0; c0 < BN; c0 += 64) {
+      if (p.N - (n0 + c0) <= 0) break;
+      uint4 w[8];
 #pragma unroll
-      for (int j = 0; j < 32; ++j) {
-        const float pr = ex2(fmaf(__uint_as_float(v[j]), LOG2E, -L2));
-        const float dj = gg * ((j == lc ? 1.f : 0.f) - pr);
-        d[j] = (valid && gg != 0.f) ? dj : 0.f;
-      }
+      for (int h = 0; h < 2; ++h) {
+        tc_ld32(taddr + c0 + 32 * h, v);
+        tc_wait_ld();
+        const int lc = id - (n0 + c0 + 32 * h);
+        float d[32];
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        if (q * 8 < ncl) {
-          uint4 w;
-          w.x = pack_bf16x2(d[q * 8 + 0], d[q * 8 + 1]);
-          w.y = pack_bf16x2(d[q * 8 + 2], d[q * 8 + 3]);
-          w.z = pack_bf16x2(d[q * 8 + 4], d[q * 8 + 5]);
-          w.w = pack_bf16x2(d[q * 8 + 6], d[q * 8 + 7]);
-          *reinterpret_cast<uint4*>(ds_row + n0 + c0 + q * 8) = w;
+        for (int j = 0; j < 32; ++j) {
+          const float pr = ex2(fmaf(__uint_as_float(v[j]), LOG2E, -L2));
+          d[j] = live ? gg * ((j == lc ? 1.f : 0.f) - pr) : 0.f;
         }
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+          w[4 * h + q] = make_uint4(pack_bf16x2(d[q * 8 + 0], d[q * 8 + 1]), pack_bf16x2(d[q * 8 + 2], d[q * 8 + 3]),
+                                    pack_bf16x2(d[q * 8 + 4], d[q * 8 + 5]), pack_bf16x2(d[q * 8 + 6], d[q * 8 + 7]));
       }
+      wo.put<false>(w, n0 + c0, mb * BM + quad * 32);     // columns >= V are clipped by the TMA
     }
   } else if constexpr (EPI == TC_EPI_E) {
     const int blk = p.blk_off + mb;
@@ -263,38 +302,35 @@ __device__ __forceinline__ void epilogue_tile(const TcArgs& p, uint32_t tmem_acc
     const int id = valid ? p.ids[grow] : -1;
     const float C2 = valid ? p.lse[grow] * LOG2E : 0.f;      // p.lse holds the shift c here
     const size_t srow = (size_t)mb * BM + r;
-    __nv_bfloat16* e_row = p.dS + srow * p.ds_ld;
     float sum = 0.f, tg = 0.f;
     bool has = false;
-    for (int c0 = 0; c0 < BN; c0 += 32) {
-      const int ncl = p.N - (n0 + c0);
-      if (ncl <= 0) break;
-      tc_ld32(taddr + c0, v);
-      tc_wait_ld();
-      float d[32];
+    for (int c0 = 0; c0 < BN; c0 += 64) {
+      if (p.N - (n0 + c0) <= 0) break;
+      uint4 w[8];
 #pragma unroll
-      for (int j = 0; j < 32; ++j) {
-        const float e = ex2(fmaf(__uint_as_float(v[j]), LOG2E, -C2));
-        d[j] = (valid && j < ncl) ? e : 0.f;
-        sum += d[j];
-      }
-      const int lc = id - (n0 + c0);
-      if (lc >= 0 && lc < 32 && lc < ncl) {
+      for (int h = 0; h < 2; ++h) {
+        const int ncl = p.N - (n0 + c0 + 32 * h);           // may be <= 0 for the second half
+        tc_ld32(taddr + c0 + 32 * h, v);
+        tc_wait_ld();
+        float d[32];
 #pragma unroll
-        for (int j = 0; j < 32; ++j) if (j == lc) tg = __uint_as_float(v[j]);
-        has = true;
-      }
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        if (q * 8 < ncl) {
-          uint4 w;
-          w.x = pack_bf16x2(d[q * 8 + 0], d[q * 8 + 1]);
-          w.y = pack_bf16x2(d[q * 8 + 2], d[q * 8 + 3]);
-          w.z = pack_bf16x2(d[q * 8 + 4], d[q * 8 + 5]);
-          w.w = pack_bf16x2(d[q * 8 + 6], d[q * 8 + 7]);
-          *reinterpret_cast<uint4*>(e_row + n0 + c0 + q * 8) = w;
+        for (int j = 0; j < 32; ++j) {
+          const float e = ex2(fmaf(__uint_as_float(v[j]), LOG2E, -C2));
+          d[j] = (valid && j < ncl) ? e : 0.f;
+          sum += d[j];
         }
+        const int lc = id - (n0 + c0 + 32 * h);
+        if (lc >= 0 && lc < 32 && lc < ncl) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) if (j == lc) tg = __uint_as_float(v[j]);
+          has = true;
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+          w[4 * h + q] = make_uint4(pack_bf16x2(d[q * 8 + 0], d[q * 8 + 1]), pack_bf16x2(d[q * 8 + 2], d[q * 8 + 3]),
+                                    pack_bf16x2(d[q * 8 + 4], d[q * 8 + 5]), pack_bf16x2(d[q * 8 + 6], d[q * 8 + 7]));
       }
+      wo.put<false>(w, n0 + c0, mb * BM + quad * 32);
     }
     p.psum[(size_t)nt * p.rows_cap + srow] = sum;
     if (has) p.tgt[srow] = tg;
@@ -323,29 +359,15 @@ __device__ __forceinline__ void epilogue_tile(const TcArgs& p, uint32_t tmem_acc
         }
       }
     }
-  } else {  // TC_EPI_DW
-    const long vrow = (long)mb * BM + r;
-    const bool valid = vrow < p.V;
-    float* out = p.dW + (size_t)vrow * p.dw_ld;
+  } else {  // TC_EPI_DW: rows >= V and columns >= H are clipped by the TMA
     for (int c0 = 0; c0 < BN; c0 += 32) {
-      const int ncl = p.N - (n0 + c0);
-      if (ncl <= 0) break;
+      if (p.N - (n0 + c0) <= 0) break;
       tc_ld32(taddr + c0, v);
       tc_wait_ld();
-      if (valid) {
+      uint4 w[8];
 #pragma unroll
-        for (int q = 0; q < 8; ++q) {
-          if (q * 4 < ncl) {
-            float4* ptr = reinterpret_cast<float4*>(out + n0 + c0 + q * 4);
-            float4 o = *ptr;
-            o.x += __uint_as_float(v[q * 4 + 0]);
-            o.y += __uint_as_float(v[q * 4 + 1]);
-            o.z += __uint_as_float(v[q * 4 + 2]);
-            o.w += __uint_as_float(v[q * 4 + 3]);
-            *ptr = o;
-          }
-        }
-      }
+      for (int q = 0; q < 8; ++q) w[q] = make_uint4(v[q * 4 + 0], v[q * 4 + 1], v[q * 4 + 2], v[q * 4 + 3]);
+      wo.put<true>(w, n0 + c0, mb * BM + quad * 32);
     }
   }
 }
@@ -353,18 +375,20 @@ __device__ __forceinline__ void epilogue_tile(const TcArgs& p, uint32_t tmem_acc
 // ---------------------------------------------------------------- the kernel
 template <int EPI>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcArgs p) {
+tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               const __grid_constant__ CUtensorMap tmOut, const TcArgs p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t bar_base = smem_base + STAGES * STAGE_BYTES;
+  const uint32_t out_base = smem_base + STAGES * STAGE_BYTES;          // 1024-aligned
+  const uint32_t bar_base = out_base + OUT_STAGE_BYTES;
   // barrier layout (8 B each): full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2]; then tmem slot, abort flag
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
   auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
   auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
   uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen_base + STAGES * STAGE_BYTES + 8 * (2 * STAGES + 4));
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen_base + STAGES * STAGE_BYTES + 8 * (2 * STAGES + 4) + 8);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen_base + STAGES * STAGE_BYTES + OUT_STAGE_BYTES + 8 * (2 * STAGES + 4));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen_base + STAGES * STAGE_BYTES + OUT_STAGE_BYTES + 8 * (2 * STAGES + 4) + 8);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -466,6 +490,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   } else {
     // ------------------------------------------------------------ epilogue warps 2..5
     const int quad = warp & 3;
+    WarpOut wo{out_base + (uint32_t)quad * 8192u, &tmOut, lane, 0};
     int acc = 0; uint32_t acc_phase = 0;
     for (int tile = blockIdx.x; tile < total; tile += gridDim.x) {
       int mb, nt;
@@ -474,11 +499,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      epilogue_tile<EPI>(p, tmem_base + (uint32_t)(acc * BN), quad, lane, mb, nt);
+      epilogue_tile<EPI>(p, tmem_base + (uint32_t)(acc * BN), quad, lane, mb, nt, wo);
       tc_fence_before();
       mbar_arrive(tempty_bar(acc));
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
+    wo.drain();      // staged stores must have left shared memory before the CTA exits
   }
 
   tc_fence_before();
@@ -522,15 +548,31 @@ bool make_tmap(CUtensorMap* tm, const void* base, long rows, long K, long ld, in
   return r == CUDA_SUCCESS;
 }
 
+// Output tile map for the staged stores: [outer, inner] elements, box = 32 rows x 128 bytes.
+bool make_out_tmap(CUtensorMap* tm, void* base, long inner, long outer, long ld, bool f32) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return false;
+  const int esz = f32 ? 4 : 2;
+  cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
+  cuuint64_t strides[1] = {(cuuint64_t)ld * esz};
+  cuuint32_t box[2] = {(cuuint32_t)(128 / esz), 32u};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(tm, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides,
+                  box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
 template <int EPI>
-cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, const TcArgs& a, int grid, cudaStream_t s) {
+cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmOut, const TcArgs& a, int grid,
+                       cudaStream_t s) {
   static bool attr_set = false;
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  tc_gemm_kernel<EPI><<<grid, NUM_THREADS, SMEM_BYTES, s>>>(tmA, tmB, a);
+  tc_gemm_kernel<EPI><<<grid, NUM_THREADS, SMEM_BYTES, s>>>(tmA, tmB, tmOut, a);
   note_launch();
   return cudaGetLastError();
 }
@@ -551,6 +593,12 @@ cudaError_t launch_tc_gemm(const TcGemm& g, cudaStream_t s) {
   CUtensorMap tmA, tmB;
   if (!make_tmap(&tmA, g.A, g.a_rows, g.K, g.a_ld, BM, a_is_mn(g.epi))) return cudaErrorInvalidValue;
   if (!make_tmap(&tmB, g.B, g.b_rows, g.K, g.b_ld, BN, b_is_mn(g.epi))) return cudaErrorInvalidValue;
+  CUtensorMap tmOut = tmA;      // unused by the LSE and DH epilogues
+  if (g.epi == TC_EPI_DS || g.epi == TC_EPI_E) {
+    if (!make_out_tmap(&tmOut, g.dS, g.N, (long)g.blk_cap * BM, g.ds_ld, false)) return cudaErrorInvalidValue;
+  } else if (g.epi == TC_EPI_DW) {
+    if (!make_out_tmap(&tmOut, g.dW, g.N, g.V, g.dw_ld, true)) return cudaErrorInvalidValue;
+  }
   TcArgs a;
   a.N = g.N; a.K = g.K; a.m_blocks_fixed = g.m_blocks; a.blk_off = g.blk_off; a.blk_cap = g.blk_cap;
   a.raster_band = g.raster_band > 0 ? g.raster_band : 16; a.rows_cap = g.rows_cap; a.V = g.V;
@@ -563,11 +611,11 @@ cudaError_t launch_tc_gemm(const TcGemm& g, cudaStream_t s) {
   const long max_tiles = (long)(g.epi == TC_EPI_DW ? g.m_blocks : g.blk_cap) * NT;
   const int grid = (int)(max_tiles < (long)tc_num_sms() ? (max_tiles > 0 ? max_tiles : 1) : tc_num_sms());
   switch (g.epi) {
-    case TC_EPI_LSE: return launch_one<TC_EPI_LSE>(tmA, tmB, a, grid, s);
-    case TC_EPI_DS: return launch_one<TC_EPI_DS>(tmA, tmB, a, grid, s);
-    case TC_EPI_DH: return launch_one<TC_EPI_DH>(tmA, tmB, a, grid, s);
-    case TC_EPI_DW: return launch_one<TC_EPI_DW>(tmA, tmB, a, grid, s);
-    case TC_EPI_E: return launch_one<TC_EPI_E>(tmA, tmB, a, grid, s);
+    case TC_EPI_LSE: return launch_one<TC_EPI_LSE>(tmA, tmB, tmOut, a, grid, s);
+    case TC_EPI_DS: return launch_one<TC_EPI_DS>(tmA, tmB, tmOut, a, grid, s);
+    case TC_EPI_DH: return launch_one<TC_EPI_DH>(tmA, tmB, tmOut, a, grid, s);
+    case TC_EPI_DW: return launch_one<TC_EPI_DW>(tmA, tmB, tmOut, a, grid, s);
+    case TC_EPI_E: return launch_one<TC_EPI_E>(tmA, tmB, tmOut, a, grid, s);
   }
   return cudaErrorInvalidValue;
 }
