@@ -10,7 +10,7 @@ namespace {
 constexpr int kRecommendedChunkRowsBf16 = 32768;
 constexpr int kRecommendedChunkRowsF32 = 2048;
 constexpr int kRasterBandFwd = 32;
-constexpr int kRasterBandBwd = 8;
+constexpr int kRasterBandBwd = 4;
 
 int check_device() {
   static int cached = -1;

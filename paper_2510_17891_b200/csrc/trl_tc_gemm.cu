@@ -18,7 +18,8 @@
 // Roles: warp 0 = TMA producer (one elected lane), warp 1 = MMA issuer (one elected lane)
 // and TMEM owner, warps 2..5 = epilogue (one TMEM lane quadrant each).  Shared-memory
 // stages are guarded by full/empty mbarriers; the 512 TMEM columns hold two 128x256 fp32
-// accumulators so the epilogue of tile i overlaps the mainloop of tile i+1.
+// accumulators: in the forward GEMMs the epilogue of tile i overlaps the mainloop of tile
+// i+1, in the gradient GEMMs both belong to one 256x256 CTA tile that shares its B operand.
 // The dS / E / dW epilogues stage 32-row x 128-byte units in swizzled shared memory and hand
 // them to the TMA (bulk tensor store / reduce-add), so global memory sees whole 128 B lines.
 // Every wait is bounded: on expiry the CTA raises TRL_ERR_TIMEOUT in the status word,
@@ -373,10 +374,24 @@ __device__ __forceinline__ void epilogue_tile(const TcArgs& p, uint32_t tmem_acc
 }
 
 // ---------------------------------------------------------------- the kernel
+// MT = 128-row M blocks per CTA tile.  The forward GEMMs (K = H, short mainloop) use MT = 1 and
+// alternate between two TMEM accumulators so the epilogue overlaps the next mainloop.  The
+// gradient GEMMs (K = V or K = rows of a chunk: long mainloop, operands streaming from HBM)
+// use MT = 2: one B tile in shared memory feeds both accumulators, which cuts the shared-memory
+// fill traffic per FLOP by a third; their epilogue is a few % of the mainloop and runs exposed.
+template <int EPI> struct TileCfg {
+  static constexpr int MT = (EPI == TC_EPI_DH || EPI == TC_EPI_DW) ? 2 : 1;
+  static constexpr int NACC = 2 / MT;                       // accumulator sets in the 512 TMEM columns
+  static constexpr int STG_BYTES = MT * A_BYTES + B_BYTES;  // 48 KB or 64 KB
+  static constexpr int NSTAGE = (STAGES * STAGE_BYTES) / STG_BYTES;   // 4 or 3
+};
+
 template <int EPI>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmOut, const TcArgs p) {
+  using Cfg = TileCfg<EPI>;
+  constexpr int MT = Cfg::MT, NACC = Cfg::NACC, NSTAGE = Cfg::NSTAGE, STG = Cfg::STG_BYTES;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t out_base = smem_base + STAGES * STAGE_BYTES;          // 1024-aligned
@@ -395,11 +410,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   // ---- problem extents (identical in every thread)
   int live = p.blk_cap;
   if (p.nblk) live = max(0, min(p.nblk[0] - p.blk_off, p.blk_cap));
-  const int MB = (EPI == TC_EPI_DW) ? p.m_blocks_fixed : live;
+  const int MB = (EPI == TC_EPI_DW) ? p.m_blocks_fixed : live;    // 128-row blocks
+  const int MS = (MB + MT - 1) / MT;                               // CTA tiles along M
   const int K = (EPI == TC_EPI_DW) ? live * BM : p.K;
   const int NT = (p.N + BN - 1) / BN;
   const int nkb = (K + BK - 1) / BK;
-  const int total = (nkb > 0) ? MB * NT : 0;
+  const int total = (nkb > 0) ? MS * NT : 0;
   if (total == 0 || (int)blockIdx.x >= total) return;
 
   if (threadIdx.x == 0) {
@@ -419,6 +435,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  auto a_row_of = [&](int mb) {
+    // forward GEMMs read hidden at the row block's own rows; the gradient GEMMs read chunk scratch
+    return (EPI == TC_EPI_LSE || EPI == TC_EPI_DS || EPI == TC_EPI_E) ? p.blk_row[p.blk_off + mb] : mb * BM;
+  };
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
@@ -426,28 +446,34 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       int stage = 0; uint32_t phase = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x) {
-        int mb, nt;
-        tile_coords(tile, MB, NT, p.raster_band, mb, nt);
-        const int a_row = (EPI == TC_EPI_LSE || EPI == TC_EPI_DS || EPI == TC_EPI_E) ? p.blk_row[p.blk_off + mb] : mb * BM;
+        int ms, nt;
+        tile_coords(tile, MS, NT, p.raster_band, ms, nt);
+        const int nm = min(MT, MB - ms * MT);                 // M blocks present in this tile (1 or 2)
         const int b_row = nt * BN;
         for (int kb = 0; kb < nkb; ++kb) {
           if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status))) break;
-          mbar_expect_tx(full_bar(stage), STAGE_BYTES);
-          const uint32_t sa = smem_base + stage * STAGE_BYTES;
-          if constexpr (a_is_mn(EPI)) {       // two 64(M) x 64(K) boxes
-            tma_load_2d(sa, &tmA, a_row, kb * BK, full_bar(stage));
-            tma_load_2d(sa + 8192, &tmA, a_row + 64, kb * BK, full_bar(stage));
-          } else {
-            tma_load_2d(sa, &tmA, kb * BK, a_row, full_bar(stage));
+          mbar_expect_tx(full_bar(stage), (uint32_t)(nm * A_BYTES + B_BYTES));
+          const uint32_t sa = smem_base + stage * STG;
+#pragma unroll
+          for (int j = 0; j < MT; ++j) {
+            if (j < nm) {
+              const int a_row = a_row_of(ms * MT + j);
+              if constexpr (a_is_mn(EPI)) {       // two 64(M) x 64(K) boxes
+                tma_load_2d(sa + j * A_BYTES, &tmA, a_row, kb * BK, full_bar(stage));
+                tma_load_2d(sa + j * A_BYTES + 8192, &tmA, a_row + 64, kb * BK, full_bar(stage));
+              } else {
+                tma_load_2d(sa + j * A_BYTES, &tmA, kb * BK, a_row, full_bar(stage));
+              }
+            }
           }
+          const uint32_t sb = sa + MT * A_BYTES;
           if constexpr (b_is_mn(EPI)) {       // four 64(N) x 64(K) boxes
 #pragma unroll
-            for (int j = 0; j < BN / 64; ++j)
-              tma_load_2d(sa + A_BYTES + j * 8192, &tmB, b_row + 64 * j, kb * BK, full_bar(stage));
+            for (int j = 0; j < BN / 64; ++j) tma_load_2d(sb + j * 8192, &tmB, b_row + 64 * j, kb * BK, full_bar(stage));
           } else {
-            tma_load_2d(sa + A_BYTES, &tmB, kb * BK, b_row, full_bar(stage));
+            tma_load_2d(sb, &tmB, kb * BK, b_row, full_bar(stage));
           }
-          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+          if (++stage == NSTAGE) { stage = 0; phase ^= 1u; }
         }
       }
       if (!ok) {   // give copies already in flight time to land before shared memory is released
@@ -463,27 +489,36 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       int acc = 0; uint32_t acc_phase = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x) {
+        int ms, nt;
+        tile_coords(tile, MS, NT, p.raster_band, ms, nt);
+        const int nm = min(MT, MB - ms * MT);
         if (!(ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, p.status))) break;
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * MT * BN);
         for (int kb = 0; kb < nkb; ++kb) {
           if (!(ok = mbar_wait(full_bar(stage), phase, abort_flag, p.status))) break;
           tc_fence_after();
-          const uint32_t sa = smem_base + stage * STAGE_BYTES;
-          const uint64_t da = a_is_mn(EPI) ? make_mnmajor_sw128_desc(sa) : make_kmajor_sw128_desc(sa);
-          const uint64_t db = b_is_mn(EPI) ? make_mnmajor_sw128_desc(sa + A_BYTES) : make_kmajor_sw128_desc(sa + A_BYTES);
+          const uint32_t sa = smem_base + stage * STG;
+          const uint32_t sb = sa + MT * A_BYTES;
+          const uint64_t db = b_is_mn(EPI) ? make_mnmajor_sw128_desc(sb) : make_kmajor_sw128_desc(sb);
           // one MMA consumes 16 k.  K-major: 32 B further along the 128 B swizzle row (+2 in the
           // >>4 address field).  MN-major: two 8-row atoms of 1024 B further (+128).
           constexpr uint64_t ka = a_is_mn(EPI) ? 128 : 2, kbs = b_is_mn(EPI) ? 128 : 2;
 #pragma unroll
-          for (int k = 0; k < BK / UMMA_K; ++k)
-            tc_mma_bf16(d_tmem, da + ka * k, db + kbs * k, idesc, (uint32_t)((kb | k) != 0));
+          for (int j = 0; j < MT; ++j) {
+            if (j < nm) {
+              const uint64_t da = a_is_mn(EPI) ? make_mnmajor_sw128_desc(sa + j * A_BYTES) : make_kmajor_sw128_desc(sa + j * A_BYTES);
+#pragma unroll
+              for (int k = 0; k < BK / UMMA_K; ++k)
+                tc_mma_bf16(d_tmem + (uint32_t)(j * BN), da + ka * k, db + kbs * k, idesc, (uint32_t)((kb | k) != 0));
+            }
+          }
           tc_commit(empty_bar(stage));
-          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+          if (++stage == NSTAGE) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
         tc_commit(tfull_bar(acc));
-        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        if (++acc == NACC) { acc = 0; acc_phase ^= 1u; }
       }
     }
     __syncwarp();
@@ -493,16 +528,19 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     WarpOut wo{out_base + (uint32_t)quad * 8192u, &tmOut, lane, 0};
     int acc = 0; uint32_t acc_phase = 0;
     for (int tile = blockIdx.x; tile < total; tile += gridDim.x) {
-      int mb, nt;
-      tile_coords(tile, MB, NT, p.raster_band, mb, nt);
+      int ms, nt;
+      tile_coords(tile, MS, NT, p.raster_band, ms, nt);
+      const int nm = min(MT, MB - ms * MT);
       bool ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.status);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      epilogue_tile<EPI>(p, tmem_base + (uint32_t)(acc * BN), quad, lane, mb, nt, wo);
+#pragma unroll
+      for (int j = 0; j < MT; ++j)
+        if (j < nm) epilogue_tile<EPI>(p, tmem_base + (uint32_t)((acc * MT + j) * BN), quad, lane, ms * MT + j, nt, wo);
       tc_fence_before();
       mbar_arrive(tempty_bar(acc));
-      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      if (++acc == NACC) { acc = 0; acc_phase ^= 1u; }
     }
     wo.drain();      // staged stores must have left shared memory before the CTA exits
   }
@@ -608,7 +646,8 @@ cudaError_t launch_tc_gemm(const TcGemm& g, cudaStream_t s) {
   a.dHidden = g.dHidden; a.dh_ld = g.dh_ld; a.dW = g.dW; a.dw_ld = g.dw_ld; a.status = g.status;
   a.psum = g.psum; a.row_scale = g.row_scale;
   const int NT = cdiv(g.N, BN);
-  const long max_tiles = (long)(g.epi == TC_EPI_DW ? g.m_blocks : g.blk_cap) * NT;
+  const int mt = (g.epi == TC_EPI_DW || g.epi == TC_EPI_DH) ? 2 : 1;
+  const long max_tiles = (long)cdiv(g.epi == TC_EPI_DW ? g.m_blocks : g.blk_cap, mt) * NT;
   const int grid = (int)(max_tiles < (long)tc_num_sms() ? (max_tiles > 0 ? max_tiles : 1) : tc_num_sms());
   switch (g.epi) {
     case TC_EPI_LSE: return launch_one<TC_EPI_LSE>(tmA, tmB, tmOut, a, grid, s);
