@@ -36,27 +36,28 @@ struct Carver {
   }
 };
 
-size_t fwd_bytes_bf16(int B, int T, int V) {
-  const size_t rows_cap = (size_t)B * cdiv(T, kRowBlock) * kRowBlock;
-  const size_t nt = cdiv(V, 256);
-  return row_blocks_bytes(B, T) + align_up(rows_cap * 4, 256) + align_up(nt * rows_cap * 8, 256);
+int rows_cap_of(int B, int T) { return cdiv(B * T, kRowBlock) * kRowBlock; }
+size_t xp_bytes(int B, int T, int H) { return align_up((size_t)rows_cap_of(B, T) * H * 2, 256); }   // packed hidden rows
+size_t fwd_extra_bf16(int B, int T, int V) {     // target logits + (max, sum-exp) partials per vocabulary tile
+  const size_t rows_cap = rows_cap_of(B, T);
+  return align_up(rows_cap * 4, 256) + align_up((size_t)cdiv(V, 256) * rows_cap * 8, 256);
 }
+size_t fwd_bytes_bf16(int B, int T, int H, int V) { return row_pack_bytes(B, T) + xp_bytes(B, T, H) + fwd_extra_bf16(B, T, V); }
 size_t fwd_bytes_f32(int B, int T, int H, int V, int R) {
-  return row_blocks_bytes(B, T) + align_up((size_t)R * H * 4, 256) + align_up((size_t)R * V * 4, 256);
+  return row_pack_bytes(B, T) + align_up((size_t)R * H * 4, 256) + align_up((size_t)R * V * 4, 256);
 }
-size_t bwd_fixed_bf16(int B, int T, int H, int V) { (void)H; (void)V; return row_blocks_bytes(B, T); }
-size_t bwd_per_rows_bf16(int H, int V, int R) {
-  return align_up((size_t)H * R * 2, 256) + align_up((size_t)R * V * 2, 256);   // gathered hidden rows + dS / E
-}
+size_t bwd_fixed_bf16(int B, int T, int H, int V) { (void)V; return row_pack_bytes(B, T) + xp_bytes(B, T, H); }
+size_t bwd_per_rows_bf16(int H, int V, int R) { (void)H; return align_up((size_t)R * V * 2, 256); }   // dS chunk
 size_t bwd_bytes_f32(int B, int T, int H, int V, int R) {
-  return row_blocks_bytes(B, T) + 2 * align_up((size_t)R * H * 4, 256) + align_up((size_t)R * V * 4, 256);
+  return row_pack_bytes(B, T) + 2 * align_up((size_t)R * H * 4, 256) + align_up((size_t)R * V * 4, 256);
 }
-int rows_cap_of(int B, int T) { return B * cdiv(T, kRowBlock) * kRowBlock; }
 size_t loss_bytes(int B, int T) { return align_up((size_t)B * pg_loss_tiles(T) * 4 * sizeof(float), 256); }
-// fused step: fixed part (row blocks, W^T, loss partials) and per-chunk part for R rows
+// fused step: fixed part (row packing, packed hidden, loss partials) and per-chunk part for R rows
+// (scaled hidden rows, E, row sums per vocabulary tile, target logits, row factors)
 size_t fused_fixed_bf16(int B, int T, int H, int V) { return bwd_fixed_bf16(B, T, H, V) + loss_bytes(B, T); }
 size_t fused_per_rows_bf16(int H, int V, int R) {
-  return bwd_per_rows_bf16(H, V, R) + align_up((size_t)cdiv(V, 256) * R * 4, 256) + 2 * align_up((size_t)R * 4, 256);
+  return align_up((size_t)H * R * 2, 256) + align_up((size_t)R * V * 2, 256) + align_up((size_t)cdiv(V, 256) * R * 4, 256) +
+         2 * align_up((size_t)R * 4, 256);
 }
 
 // largest multiple of 128 rows (<= cap) whose scratch fits into `avail` bytes
@@ -76,7 +77,7 @@ size_t ws_bytes(int which, int B, int T, int H, int V, trl_dtype dt, bool minimu
   const int cap = rows_cap_of(B, T);
   switch (which) {
     case TRL_CALL_TOKEN_LOGPROBS:
-      if (dt == TRL_BF16) return fwd_bytes_bf16(B, T, V);
+      if (dt == TRL_BF16) return fwd_bytes_bf16(B, T, H, V);
       return fwd_bytes_f32(B, T, H, V, minimum ? kRowBlock : (cap < kRecommendedChunkRowsF32 ? cap : kRecommendedChunkRowsF32));
     case TRL_CALL_PG_LOSS_FWD:
       return align_up((size_t)B * pg_loss_tiles(T) * 4 * sizeof(float), 256);
@@ -90,7 +91,7 @@ size_t ws_bytes(int which, int B, int T, int H, int V, trl_dtype dt, bool minimu
       if (dt == TRL_BF16) {
         const int R = minimum ? kRowBlock : (cap < kRecommendedChunkRowsBf16 ? cap : kRecommendedChunkRowsBf16);
         // the forward workspace is appended for the lse_hint == NULL case
-        return fused_fixed_bf16(B, T, H, V) + fused_per_rows_bf16(H, V, R) + fwd_bytes_bf16(B, T, V);
+        return fused_fixed_bf16(B, T, H, V) + fused_per_rows_bf16(H, V, R) + fwd_extra_bf16(B, T, V);
       }
       size_t a = ws_bytes(TRL_CALL_TOKEN_LOGPROBS, B, T, H, V, dt, minimum);
       size_t b = ws_bytes(TRL_CALL_PG_LOSS_BWD, B, T, H, V, dt, minimum);
@@ -146,17 +147,19 @@ int trl_token_logprobs(const void* hidden, const void* W, const int32_t* ids, co
   const int cap_rows = rows_cap_of(B, T);
 
   Carver cv(workspace);
-  RowBlocks rb = carve_row_blocks(cv.take<char>(row_blocks_bytes(B, T)), B, T);
-  launch_build_row_blocks(len, B, T, rb, status_dev, s);
+  RowPack rb = carve_row_pack(cv.take<char>(row_pack_bytes(B, T)), B, T);
+  launch_build_row_pack(len, B, T, rb, status_dev, s);
 
   if (dt == TRL_BF16) {
     const int nt = cdiv(V, 256);
+    __nv_bfloat16* Xp = cv.take<__nv_bfloat16>((size_t)cap_rows * H);
     float* tgt = cv.take<float>(cap_rows);
     float2* partials = cv.take<float2>((size_t)nt * cap_rows);
+    launch_pack_rows_bf16((const __nv_bfloat16*)hidden, Xp, H, cap_rows, rb, 0, 0, nullptr, s);
     TcGemm g;
     memset(&g, 0, sizeof(g));
     g.epi = TC_EPI_LSE;
-    g.A = hidden; g.a_rows = (long)B * T; g.a_ld = H;
+    g.A = Xp; g.a_rows = cap_rows; g.a_ld = H;
     g.B = W; g.b_rows = V; g.b_ld = H;
     g.K = H; g.N = V;
     g.rb = rb; g.blk_off = 0; g.blk_cap = rb.cap; g.raster_band = kRasterBandFwd;
@@ -164,7 +167,7 @@ int trl_token_logprobs(const void* hidden, const void* W, const int32_t* ids, co
     TRL_CUDA_OK(launch_tc_gemm(g, s));
     launch_merge_lse(partials, tgt, nt, cap_rows, rb, ids, len, B, T, V, logp, lse, status_dev, s);
   } else {
-    const size_t avail = workspace_bytes - row_blocks_bytes(B, T);
+    const size_t avail = workspace_bytes - row_pack_bytes(B, T);
     const int R = fit_rows(avail, cap_rows < kRecommendedChunkRowsF32 ? cap_rows : kRecommendedChunkRowsF32,
                            [&](int r) { return align_up((size_t)r * H * 4, 256) + align_up((size_t)r * V * 4, 256); });
     if (R < kRowBlock) return TRL_ERR_WORKSPACE_TOO_SMALL;
@@ -226,8 +229,8 @@ int trl_pg_loss_bwd(const void* hidden, const void* W, const int32_t* ids, const
   const size_t N = (size_t)B * T;
 
   Carver cv(workspace);
-  RowBlocks rb = carve_row_blocks(cv.take<char>(row_blocks_bytes(B, T)), B, T);
-  launch_build_row_blocks(len, B, T, rb, status_dev, s);
+  RowPack rb = carve_row_pack(cv.take<char>(row_pack_bytes(B, T)), B, T);
+  launch_build_row_pack(len, B, T, rb, status_dev, s);
   TRL_CUDA_OK(cudaMemsetAsync(dW, 0, (size_t)V * H * sizeof(float), s));
 
   if (dt == TRL_BF16) {
@@ -236,18 +239,18 @@ int trl_pg_loss_bwd(const void* hidden, const void* W, const int32_t* ids, const
     const int R = fit_rows(avail, cap_rows < kRecommendedChunkRowsBf16 ? cap_rows : kRecommendedChunkRowsBf16,
                            [&](int r) { return bwd_per_rows_bf16(H, V, r); });
     if (R < kRowBlock) return TRL_ERR_WORKSPACE_TOO_SMALL;
-    __nv_bfloat16* Xs = cv.take<__nv_bfloat16>((size_t)H * R);
+    __nv_bfloat16* Xp = cv.take<__nv_bfloat16>((size_t)cap_rows * H);
     __nv_bfloat16* dS = cv.take<__nv_bfloat16>((size_t)R * V);
+    launch_pack_rows_bf16((const __nv_bfloat16*)hidden, Xp, H, cap_rows, rb, 0, 0, nullptr, s);
     const int CB = R / kRowBlock;
     for (int blk_off = 0; blk_off < rb.cap; blk_off += CB) {
-      launch_gather_rows_bf16((const __nv_bfloat16*)hidden, Xs, H, R, rb, blk_off, nullptr, s);
       TcGemm a;
       memset(&a, 0, sizeof(a));
       a.rb = rb; a.blk_off = blk_off; a.blk_cap = CB; a.status = status_dev;
       // dS chunk = g (onehot - softmax), from a recomputed logits tile
       TcGemm ds = a;
       ds.epi = TC_EPI_DS; ds.raster_band = kRasterBandFwd;
-      ds.A = hidden; ds.a_rows = (long)N; ds.a_ld = H; ds.B = W; ds.b_rows = V; ds.b_ld = H; ds.K = H; ds.N = V;
+      ds.A = Xp; ds.a_rows = cap_rows; ds.a_ld = H; ds.B = W; ds.b_rows = V; ds.b_ld = H; ds.K = H; ds.N = V;
       ds.ids = ids; ds.lse = lse; ds.g = g; ds.dS = dS; ds.ds_ld = V;
       TRL_CUDA_OK(launch_tc_gemm(ds, s));
       // dHidden rows of the chunk = dS W   (W read as an N-contiguous operand)
@@ -256,16 +259,18 @@ int trl_pg_loss_bwd(const void* hidden, const void* W, const int32_t* ids, const
       dh.A = dS; dh.a_rows = R; dh.a_ld = V; dh.B = W; dh.b_rows = H; dh.b_ld = H; dh.K = V; dh.N = H;
       dh.dHidden = (__nv_bfloat16*)dHidden; dh.dh_ld = H;
       TRL_CUDA_OK(launch_tc_gemm(dh, s));
-      // dW += dS^T hidden   (both operands M/N-contiguous: dS [R,V] and the gathered rows [R,H])
+      // dW += dS^T hidden   (both operands M/N-contiguous: dS [R,V] and the chunk's packed rows [.,H])
       TcGemm dw = a;
       dw.epi = TC_EPI_DW; dw.raster_band = kRasterBandBwd;
-      dw.A = dS; dw.a_rows = V; dw.a_ld = V; dw.B = Xs; dw.b_rows = H; dw.b_ld = H; dw.K = R; dw.N = H;
+      dw.A = dS; dw.a_rows = V; dw.a_ld = V; dw.K = R; dw.N = H;
+      dw.B = Xp + (size_t)blk_off * kRowBlock * H; dw.b_rows = H; dw.b_ld = H;
+      dw.b_k = cap_rows - blk_off * kRowBlock < R ? cap_rows - blk_off * kRowBlock : R;
       dw.m_blocks = cdiv(V, kRowBlock); dw.dW = dW; dw.dw_ld = H; dw.V = V;
       TRL_CUDA_OK(launch_tc_gemm(dw, s));
     }
   } else {
     TRL_CUDA_OK(cudaMemsetAsync(dHidden, 0, N * H * 4, s));
-    const size_t avail = workspace_bytes - row_blocks_bytes(B, T);
+    const size_t avail = workspace_bytes - row_pack_bytes(B, T);
     const int R = fit_rows(avail, cap_rows < kRecommendedChunkRowsF32 ? cap_rows : kRecommendedChunkRowsF32,
                            [&](int r) { return 2 * align_up((size_t)r * H * 4, 256) + align_up((size_t)r * V * 4, 256); });
     if (R < kRowBlock) return TRL_ERR_WORKSPACE_TOO_SMALL;
@@ -318,7 +323,7 @@ int trl_pg_step_fused(const void* hidden, const void* W, const int32_t* ids, con
   const int cap_rows = rows_cap_of(B, T);
   const size_t N = (size_t)B * T;
   const int nt = cdiv(V, 256);
-  const size_t fwd_extra = lse_hint ? 0 : fwd_bytes_bf16(B, T, V);
+  const size_t fwd_extra = lse_hint ? 0 : fwd_extra_bf16(B, T, V);
   if (workspace_bytes < fused_fixed_bf16(B, T, H, V) + fwd_extra + fused_per_rows_bf16(H, V, kRowBlock))
     return TRL_ERR_WORKSPACE_TOO_SMALL;
   const size_t avail = workspace_bytes - fused_fixed_bf16(B, T, H, V) - fwd_extra;
@@ -327,7 +332,8 @@ int trl_pg_step_fused(const void* hidden, const void* W, const int32_t* ids, con
   if (R < kRowBlock) return TRL_ERR_WORKSPACE_TOO_SMALL;
 
   Carver cv(workspace);
-  RowBlocks rb = carve_row_blocks(cv.take<char>(row_blocks_bytes(B, T)), B, T);
+  RowPack rb = carve_row_pack(cv.take<char>(row_pack_bytes(B, T)), B, T);
+  __nv_bfloat16* Xp = cv.take<__nv_bfloat16>((size_t)cap_rows * H);
   float* loss_partials = cv.take<float>((size_t)B * pg_loss_tiles(T) * 4);
   __nv_bfloat16* Xs = cv.take<__nv_bfloat16>((size_t)H * R);
   __nv_bfloat16* E = cv.take<__nv_bfloat16>((size_t)R * V);
@@ -335,10 +341,11 @@ int trl_pg_step_fused(const void* hidden, const void* W, const int32_t* ids, con
   float* tgt = cv.take<float>(R);
   float* neg_alpha = cv.take<float>(R);
 
-  launch_build_row_blocks(len, B, T, rb, status_dev, s);
+  launch_build_row_pack(len, B, T, rb, status_dev, s);
   TRL_CUDA_OK(cudaMemsetAsync(dW, 0, (size_t)V * H * sizeof(float), s));
   TRL_CUDA_OK(cudaMemsetAsync(dHidden, 0, N * H * 2, s));
   launch_zero_padded_f32(logp, lse, len, B, T, s);
+  launch_pack_rows_bf16((const __nv_bfloat16*)hidden, Xp, H, cap_rows, rb, 0, 0, nullptr, s);
 
   TcGemm base;
   memset(&base, 0, sizeof(base));
@@ -350,7 +357,7 @@ int trl_pg_step_fused(const void* hidden, const void* W, const int32_t* ids, con
     float2* partials = cv.take<float2>((size_t)nt * cap_rows);
     TcGemm f = base;
     f.epi = TC_EPI_LSE; f.raster_band = kRasterBandFwd;
-    f.A = hidden; f.a_rows = (long)N; f.a_ld = H; f.B = W; f.b_rows = V; f.b_ld = H; f.K = H; f.N = V;
+    f.A = Xp; f.a_rows = cap_rows; f.a_ld = H; f.B = W; f.b_rows = V; f.b_ld = H; f.K = H; f.N = V;
     f.blk_off = 0; f.blk_cap = rb.cap; f.ids = ids; f.partials = partials; f.tgt = tgt_all; f.rows_cap = cap_rows;
     TRL_CUDA_OK(launch_tc_gemm(f, s));
     launch_merge_lse(partials, tgt_all, nt, cap_rows, rb, ids, len, B, T, V, logp, lse, status_dev, s);
@@ -364,13 +371,13 @@ int trl_pg_step_fused(const void* hidden, const void* W, const int32_t* ids, con
     // forward tile -> E = exp(z - c), row sums, sampled token's logit
     TcGemm e = a;
     e.epi = TC_EPI_E; e.raster_band = kRasterBandFwd;
-    e.A = hidden; e.a_rows = (long)N; e.a_ld = H; e.B = W; e.b_rows = V; e.b_ld = H; e.K = H; e.N = V;
+    e.A = Xp; e.a_rows = cap_rows; e.a_ld = H; e.B = W; e.b_rows = V; e.b_ld = H; e.K = H; e.N = V;
     e.ids = ids; e.lse = hint; e.dS = E; e.ds_ld = V; e.psum = psum; e.tgt = tgt; e.rows_cap = R;
     TRL_CUDA_OK(launch_tc_gemm(e, s));
     FusedMergeArgs m{psum, tgt, nt, R, rb, blk_off, ids, len, hint, old_logp, adv, seg, P, G, T, V, cfg,
                      logp, lse, g, neg_alpha, E, status_dev};
     launch_fused_merge(m, s);
-    launch_gather_rows_bf16((const __nv_bfloat16*)hidden, Xs, H, R, rb, blk_off, neg_alpha, s);
+    launch_pack_rows_bf16(Xp, Xs, H, R, rb, blk_off * kRowBlock, 1, neg_alpha, s);
     // dHidden rows = neg_alpha * (E' W)
     TcGemm dh = a;
     dh.epi = TC_EPI_DH; dh.raster_band = kRasterBandBwd;

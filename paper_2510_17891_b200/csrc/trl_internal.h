@@ -18,20 +18,21 @@ unsigned long long launches_so_far();
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline int cdiv(int a, int b) { return (a + b - 1) / b; }
 
-// Row blocks: every rollout's valid rows [b*T, b*T+len) are cut into blocks of <=128
-// consecutive rows.  Built on the device from `len` (no host round trip).
-struct RowBlocks {
-  int* nblk;       // [1]   number of live blocks
-  int* blk_first;  // [B+1] first block of each rollout (exclusive prefix sum)
-  int* blk_row;    // [cap] global row index of the block's first row
-  int* blk_n;      // [cap] valid rows in the block (1..128)
-  int cap;         // B * ceil(T/128): upper bound on nblk
+// Row packing: the valid rows of all rollouts, in order, get consecutive packed indices
+// q = row_first[b] + t (t < len[b]); 128 consecutive packed rows form one row block (one
+// accumulator tile).  Built on the device from `len` (no host round trip).
+struct RowPack {
+  int* nblk;       // [1]     ceil(n_rows / 128)
+  int* n_rows;     // [1]     number of valid rows
+  int* row_first;  // [B+1]   packed index of each rollout's first row (exclusive prefix sum of len)
+  int* rowmap;     // [cap*128] packed row -> global row b*T + t (defined for q < n_rows)
+  int cap;         // ceil(B*T / 128): upper bound on nblk
 };
-size_t row_blocks_bytes(int B, int T);
-RowBlocks carve_row_blocks(void* base, int B, int T);
+size_t row_pack_bytes(int B, int T);
+RowPack carve_row_pack(void* base, int B, int T);
 
 // ---- small kernels (trl_small_kernels.cu) ------------------------------------------
-void launch_build_row_blocks(const int32_t* len, int B, int T, RowBlocks rb, int32_t* status, cudaStream_t s);
+void launch_build_row_pack(const int32_t* len, int B, int T, RowPack rb, int32_t* status, cudaStream_t s);
 void launch_hrd_advantages(const float* r_plan, const float* r_code, const int32_t* len, const int32_t* bnd,
                            int P, int G, int T, int adv_mode, float* A_plan, float* A_code, uint8_t* seg,
                            float* adv, int32_t* n_plan, int32_t* n_code, int64_t* n_valid, int32_t* status,
@@ -41,17 +42,18 @@ void launch_pg_loss(const float* logp, const float* old_logp, const float* adv, 
                     const int32_t* len, int P, int G, int T, trl_pg_config cfg, float* loss, float* g,
                     float* stats, float* partials, cudaStream_t s);
 // merge per-vocabulary-tile (max, sumexp) partials into lse / logp and scatter to global rows
-void launch_merge_lse(const float2* partials, const float* tgt, int n_tiles, int rows_cap, RowBlocks rb,
+void launch_merge_lse(const float2* partials, const float* tgt, int n_tiles, int rows_cap, RowPack rb,
                       const int32_t* ids, const int32_t* len, int B, int T, int V, float* logp, float* lse,
                       int32_t* status, cudaStream_t s);
-// Xs[r, :] = hidden[row(blk_off*128 + r), :] for the live rows of a chunk (times
-// row_scale[r] when given), 0 elsewhere
-void launch_gather_rows_bf16(const __nv_bfloat16* hidden, __nv_bfloat16* Xs, int H, int R, RowBlocks rb,
-                             int blk_off, const float* row_scale, cudaStream_t s);
+// out[r, :] = src[row, :] (times row_scale[r] when given) for r < R, where the packed row is
+// q = q_off + r and row = rowmap[q] (from_packed = 0: src is the caller's [N,H] tensor) or
+// row = q (from_packed = 1: src is already packed); rows q >= n_rows are written as zeros.
+void launch_pack_rows_bf16(const __nv_bfloat16* src, __nv_bfloat16* out, int H, int R, RowPack rb, int q_off,
+                           int from_packed, const float* row_scale, cudaStream_t s);
 // Chunk-local finish of the fused step: lse = c + log(sum_k psum), logp, g = d loss/d logp,
 // the per-row factor -g exp(c - lse) for the gradient GEMMs, and the one-hot fix of E / E^T.
 struct FusedMergeArgs {
-  const float* psum; const float* tgt; int n_tiles; int R; RowBlocks rb; int blk_off;
+  const float* psum; const float* tgt; int n_tiles; int R; RowPack rb; int blk_off;
   const int32_t* ids; const int32_t* len; const float* hint; const float* old_logp; const float* adv;
   const uint8_t* seg; int P, G, T, V; trl_pg_config cfg;
   float* logp; float* lse; float* g; float* neg_alpha;
@@ -60,12 +62,12 @@ struct FusedMergeArgs {
 };
 void launch_fused_merge(const FusedMergeArgs& a, cudaStream_t s);
 // fp32 path helpers
-void launch_pack_rows_f32(const float* hidden, float* Xp, int H, int R, RowBlocks rb, int blk_off, cudaStream_t s);
-void launch_row_lse_f32(const float* S, int V, int R, RowBlocks rb, int blk_off, const int32_t* ids,
+void launch_pack_rows_f32(const float* hidden, float* Xp, int H, int R, RowPack rb, int blk_off, cudaStream_t s);
+void launch_row_lse_f32(const float* S, int V, int R, RowPack rb, int blk_off, const int32_t* ids,
                         float* logp, float* lse, int32_t* status, cudaStream_t s);
-void launch_ds_inplace_f32(float* S, int V, int R, RowBlocks rb, int blk_off, const int32_t* ids,
+void launch_ds_inplace_f32(float* S, int V, int R, RowPack rb, int blk_off, const int32_t* ids,
                            const float* lse, const float* g, cudaStream_t s);
-void launch_scatter_rows_f32(const float* dHp, float* dHidden, int H, int R, RowBlocks rb, int blk_off, cudaStream_t s);
+void launch_scatter_rows_f32(const float* dHp, float* dHidden, int H, int R, RowPack rb, int blk_off, cudaStream_t s);
 void launch_zero_padded_f32(float* a, float* b, const int32_t* len, int B, int T, cudaStream_t s);
 
 // ---- fp32 CUDA-core GEMM (trl_simt_gemm.cu) ----------------------------------------
@@ -91,10 +93,11 @@ struct TcGemm {
   // operand (B of DH; A and B of DW): stored [K, rows], pitch ld.
   const void* A; long a_rows; long a_ld;
   const void* B; long b_rows; long b_ld;
+  long b_k;                                  // K extent of B's storage if it differs from K (0: same)
   int K;                                     // host K extent (TC_EPI_DW: K = 128 * live blocks of the chunk)
   int N;                                     // GEMM N extent = b_rows that are meaningful
   int m_blocks;                              // TC_EPI_DW: fixed number of 128-row blocks of A; others: from row blocks
-  RowBlocks rb; int blk_off, blk_cap;        // chunk of row blocks
+  RowPack rb; int blk_off, blk_cap;        // chunk of row blocks
   int raster_band;
   // epilogue arguments
   const int32_t* ids; const float* lse; const float* g;

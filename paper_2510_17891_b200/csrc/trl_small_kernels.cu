@@ -15,26 +15,28 @@ __device__ __forceinline__ void flag_status(int32_t* status, int code) {
   if (status) atomicOr(status, 1 << code);
 }
 
-size_t row_blocks_bytes(int B, int T) {
-  size_t cap = (size_t)B * cdiv(T, kRowBlock);
-  return align_up((1 + (size_t)B + 1 + 2 * cap) * sizeof(int), 256);
+size_t row_pack_bytes(int B, int T) {
+  const size_t cap_rows = (size_t)cdiv(B * T, kRowBlock) * kRowBlock;
+  return align_up((2 + (size_t)B + 1 + cap_rows) * sizeof(int), 256);
 }
 
-RowBlocks carve_row_blocks(void* base, int B, int T) {
-  RowBlocks rb;
+RowPack carve_row_pack(void* base, int B, int T) {
+  RowPack rb;
   int* p = (int*)base;
-  rb.cap = B * cdiv(T, kRowBlock);
+  rb.cap = cdiv(B * T, kRowBlock);
   rb.nblk = p;
-  rb.blk_first = p + 1;
-  rb.blk_row = p + 1 + (B + 1);
-  rb.blk_n = rb.blk_row + rb.cap;
+  rb.n_rows = p + 1;
+  rb.row_first = p + 2;
+  rb.rowmap = p + 2 + (B + 1);
   return rb;
 }
 
-// One CTA.  Pass 1: per-thread serial counts over a contiguous slice of rollouts, block
-// scan over slices; pass 2: each rollout writes its blocks.
-__global__ void build_row_blocks_kernel(const int32_t* __restrict__ len, int B, int T, RowBlocks rb,
-                                        int32_t* status) {
+__device__ __forceinline__ long packed_to_global(const RowPack& rb, int q) {
+  return q < rb.n_rows[0] ? (long)rb.rowmap[q] : -1;
+}
+
+// One CTA: exclusive prefix sum of the (clamped) lengths.
+__global__ void build_row_pack_kernel(const int32_t* __restrict__ len, int B, int T, RowPack rb, int32_t* status) {
   __shared__ int s_sum[1024];
   const int tid = threadIdx.x, nt = blockDim.x;
   const int per = (B + nt - 1) / nt;
@@ -44,34 +46,41 @@ __global__ void build_row_blocks_kernel(const int32_t* __restrict__ len, int B, 
   for (int b = b0; b < b1; ++b) {
     int L = len[b];
     if (L < 0 || L > T) { bad = true; L = max(0, min(L, T)); }
-    cnt += (L + kRowBlock - 1) / kRowBlock;
+    cnt += L;
   }
   if (bad) flag_status(status, TRL_ERR_BAD_INDEX);
   s_sum[tid] = cnt;
   __syncthreads();
-  // inclusive Hillis-Steele scan
-  for (int off = 1; off < nt; off <<= 1) {
+  for (int off = 1; off < nt; off <<= 1) {      // inclusive Hillis-Steele scan
     int v = (tid >= off) ? s_sum[tid - off] : 0;
     __syncthreads();
     s_sum[tid] += v;
     __syncthreads();
   }
   int first = s_sum[tid] - cnt;
-  if (tid == nt - 1) { rb.nblk[0] = s_sum[tid]; rb.blk_first[B] = s_sum[tid]; }
+  if (tid == nt - 1) {
+    rb.n_rows[0] = s_sum[tid];
+    rb.nblk[0] = (s_sum[tid] + kRowBlock - 1) / kRowBlock;
+    rb.row_first[B] = s_sum[tid];
+  }
   for (int b = b0; b < b1; ++b) {
-    int L = max(0, min(len[b], T));
-    rb.blk_first[b] = first;
-    int nb = (L + kRowBlock - 1) / kRowBlock;
-    for (int i = 0; i < nb; ++i) {
-      rb.blk_row[first + i] = b * T + i * kRowBlock;
-      rb.blk_n[first + i] = min(kRowBlock, L - i * kRowBlock);
-    }
-    first += nb;
+    rb.row_first[b] = first;
+    first += max(0, min(len[b], T));
   }
 }
 
-void launch_build_row_blocks(const int32_t* len, int B, int T, RowBlocks rb, int32_t* status, cudaStream_t s) {
-  build_row_blocks_kernel<<<1, 1024, 0, s>>>(len, B, T, rb, status);
+__global__ void __launch_bounds__(256) fill_rowmap_kernel(const int32_t* __restrict__ len, int B, int T, RowPack rb) {
+  const size_t n = (size_t)blockIdx.x * 256 + threadIdx.x;
+  if (n >= (size_t)B * T) return;
+  const int b = (int)(n / T), t = (int)(n % T);
+  if (t < max(0, min(len[b], T))) rb.rowmap[rb.row_first[b] + t] = (int)n;
+}
+
+void launch_build_row_pack(const int32_t* len, int B, int T, RowPack rb, int32_t* status, cudaStream_t s) {
+  build_row_pack_kernel<<<1, 1024, 0, s>>>(len, B, T, rb, status);
+  note_launch();
+  const size_t N = (size_t)B * T;
+  fill_rowmap_kernel<<<(unsigned)((N + 255) / 256), 256, 0, s>>>(len, B, T, rb);
   note_launch();
 }
 
@@ -274,7 +283,7 @@ void launch_pg_loss(const float* logp, const float* old_logp, const float* adv, 
 // ------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) merge_lse_kernel(const float2* __restrict__ partials,
                                                         const float* __restrict__ tgt, int n_tiles, int rows_cap,
-                                                        RowBlocks rb, const int32_t* __restrict__ ids,
+                                                        RowPack rb, const int32_t* __restrict__ ids,
                                                         const int32_t* __restrict__ len, int B, int T, int V,
                                                         float* __restrict__ logp, float* __restrict__ lse,
                                                         int32_t* status) {
@@ -284,7 +293,7 @@ __global__ void __launch_bounds__(256) merge_lse_kernel(const float2* __restrict
   const int L = max(0, min(len[b], T));
   float out_lp = 0.f, out_lse = 0.f;
   if (t < L) {
-    const size_t prow = (size_t)(rb.blk_first[b] + t / kRowBlock) * kRowBlock + (t % kRowBlock);
+    const size_t prow = (size_t)rb.row_first[b] + t;
     float M = -INFINITY;
     for (int k = 0; k < n_tiles; ++k) M = fmaxf(M, partials[(size_t)k * rows_cap + prow].x);
     float l = 0.f;
@@ -301,7 +310,7 @@ __global__ void __launch_bounds__(256) merge_lse_kernel(const float2* __restrict
   lse[n] = out_lse;
 }
 
-void launch_merge_lse(const float2* partials, const float* tgt, int n_tiles, int rows_cap, RowBlocks rb,
+void launch_merge_lse(const float2* partials, const float* tgt, int n_tiles, int rows_cap, RowPack rb,
                       const int32_t* ids, const int32_t* len, int B, int T, int V, float* logp, float* lse,
                       int32_t* status, cudaStream_t s) {
   const size_t N = (size_t)B * T;
@@ -311,41 +320,43 @@ void launch_merge_lse(const float2* partials, const float* tgt, int n_tiles, int
 }
 
 // ------------------------------------------------------------------------------------
-// Gathered (and optionally scaled) hidden rows of a chunk: the B operand of dW = dS^T hidden.
-// One CTA per scratch row; 16-byte loads and stores.
+// Row packing / gathering in bf16 (one CTA per output row, 16-byte loads and stores): the
+// packed copy of hidden that the forward GEMMs read, and the scaled chunk rows that are the
+// B operand of dW = dS^T hidden in the fused step.
 // ------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(128) gather_rows_bf16_kernel(const __nv_bfloat16* __restrict__ hidden,
-                                                               __nv_bfloat16* __restrict__ Xs, int H, int R,
-                                                               RowBlocks rb, int blk_off,
-                                                               const float* __restrict__ row_scale) {
+__global__ void __launch_bounds__(128) pack_rows_bf16_kernel(const __nv_bfloat16* __restrict__ src,
+                                                             __nv_bfloat16* __restrict__ out, int H, int R, RowPack rb,
+                                                             int q_off, int from_packed,
+                                                             const float* __restrict__ row_scale) {
   const int r = blockIdx.x;
-  const int blk = blk_off + r / kRowBlock;
-  const int lr = r % kRowBlock;
-  const bool live = blk < rb.nblk[0] && lr < rb.blk_n[blk];
-  uint4* dst = reinterpret_cast<uint4*>(Xs + (size_t)r * H);
-  if (!live) {
+  const int q = q_off + r;
+  const int n_rows = rb.n_rows[0];
+  if (q >= rb.nblk[0] * kRowBlock) return;          // beyond the last live block: never read
+  uint4* dst = reinterpret_cast<uint4*>(out + (size_t)r * H);
+  if (q >= n_rows) {
     for (int i = threadIdx.x; i < H / 8; i += 128) dst[i] = make_uint4(0, 0, 0, 0);
     return;
   }
-  const uint4* src = reinterpret_cast<const uint4*>(hidden + ((size_t)rb.blk_row[blk] + lr) * H);
+  const size_t row = from_packed ? (size_t)q : (size_t)rb.rowmap[q];
+  const uint4* s4 = reinterpret_cast<const uint4*>(src + row * H);
   const float sc = row_scale ? row_scale[r] : 1.0f;
   for (int i = threadIdx.x; i < H / 8; i += 128) {
-    uint4 x = src[i];
+    uint4 x = s4[i];
     if (row_scale) {
       __nv_bfloat162* h2 = reinterpret_cast<__nv_bfloat162*>(&x);
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        float2 f = __bfloat1622float2(h2[q]);
-        h2[q] = __floats2bfloat162_rn(f.x * sc, f.y * sc);
+      for (int k = 0; k < 4; ++k) {
+        float2 f = __bfloat1622float2(h2[k]);
+        h2[k] = __floats2bfloat162_rn(f.x * sc, f.y * sc);
       }
     }
     dst[i] = x;
   }
 }
 
-void launch_gather_rows_bf16(const __nv_bfloat16* hidden, __nv_bfloat16* Xs, int H, int R, RowBlocks rb, int blk_off,
-                             const float* row_scale, cudaStream_t s) {
-  gather_rows_bf16_kernel<<<R, 128, 0, s>>>(hidden, Xs, H, R, rb, blk_off, row_scale);
+void launch_pack_rows_bf16(const __nv_bfloat16* src, __nv_bfloat16* out, int H, int R, RowPack rb, int q_off,
+                           int from_packed, const float* row_scale, cudaStream_t s) {
+  pack_rows_bf16_kernel<<<R, 128, 0, s>>>(src, out, H, R, rb, q_off, from_packed, row_scale);
   note_launch();
 }
 
@@ -359,11 +370,10 @@ void launch_gather_rows_bf16(const __nv_bfloat16* hidden, __nv_bfloat16* Xs, int
 __global__ void __launch_bounds__(128) fused_merge_kernel(FusedMergeArgs a) {
   const int r = blockIdx.x * 128 + threadIdx.x;
   if (r >= a.R) return;
-  const int blk = a.blk_off + r / kRowBlock;
-  if (blk >= a.rb.nblk[0]) return;
-  const int lr = r % kRowBlock;
-  if (lr >= a.rb.blk_n[blk]) { a.neg_alpha[r] = 0.f; return; }
-  const size_t n = (size_t)a.rb.blk_row[blk] + lr;
+  const int q = a.blk_off * kRowBlock + r;
+  if (q >= a.rb.nblk[0] * kRowBlock) return;
+  if (q >= a.rb.n_rows[0]) { a.neg_alpha[r] = 0.f; return; }
+  const size_t n = (size_t)a.rb.rowmap[q];
   const int b = (int)(n / a.T);
   float sum = 0.f;
   for (int k = 0; k < a.n_tiles; ++k) sum += a.psum[(size_t)k * a.R + r];
@@ -402,20 +412,17 @@ void launch_fused_merge(const FusedMergeArgs& a, cudaStream_t s) {
 // ------------------------------------------------------------------------------------
 // fp32 path helpers.  Scratch row r of a chunk is (block blk_off + r/128, lane r%128).
 // ------------------------------------------------------------------------------------
-__device__ __forceinline__ long scratch_row_to_global(const RowBlocks& rb, int blk_off, int r) {
-  const int blk = blk_off + r / kRowBlock;
-  if (blk >= rb.nblk[0]) return -1;
-  const int lr = r % kRowBlock;
-  return lr < rb.blk_n[blk] ? (long)rb.blk_row[blk] + lr : -1;
+__device__ __forceinline__ long scratch_row_to_global(const RowPack& rb, int blk_off, int r) {
+  return packed_to_global(rb, blk_off * kRowBlock + r);
 }
 
 __global__ void pack_rows_f32_kernel(const float* __restrict__ hidden, float* __restrict__ Xp, int H, int R,
-                                     RowBlocks rb, int blk_off) {
+                                     RowPack rb, int blk_off) {
   const int r = blockIdx.x;
   const long n = scratch_row_to_global(rb, blk_off, r);
   for (int h = threadIdx.x; h < H; h += blockDim.x) Xp[(size_t)r * H + h] = n >= 0 ? hidden[(size_t)n * H + h] : 0.f;
 }
-void launch_pack_rows_f32(const float* hidden, float* Xp, int H, int R, RowBlocks rb, int blk_off, cudaStream_t s) {
+void launch_pack_rows_f32(const float* hidden, float* Xp, int H, int R, RowPack rb, int blk_off, cudaStream_t s) {
   pack_rows_f32_kernel<<<R, 128, 0, s>>>(hidden, Xp, H, R, rb, blk_off);
   note_launch();
 }
@@ -434,7 +441,7 @@ __device__ __forceinline__ float block_reduce(float v, bool is_max, float* sh) {
   return r;
 }
 
-__global__ void __launch_bounds__(256) row_lse_f32_kernel(const float* __restrict__ S, int V, int R, RowBlocks rb,
+__global__ void __launch_bounds__(256) row_lse_f32_kernel(const float* __restrict__ S, int V, int R, RowPack rb,
                                                           int blk_off, const int32_t* __restrict__ ids,
                                                           float* __restrict__ logp, float* __restrict__ lse,
                                                           int32_t* status) {
@@ -457,13 +464,13 @@ __global__ void __launch_bounds__(256) row_lse_f32_kernel(const float* __restric
     else { logp[n] = 0.f; flag_status(status, TRL_ERR_BAD_INDEX); }
   }
 }
-void launch_row_lse_f32(const float* S, int V, int R, RowBlocks rb, int blk_off, const int32_t* ids, float* logp,
+void launch_row_lse_f32(const float* S, int V, int R, RowPack rb, int blk_off, const int32_t* ids, float* logp,
                         float* lse, int32_t* status, cudaStream_t s) {
   row_lse_f32_kernel<<<R, 256, 0, s>>>(S, V, R, rb, blk_off, ids, logp, lse, status);
   note_launch();
 }
 
-__global__ void __launch_bounds__(256) ds_inplace_f32_kernel(float* __restrict__ S, int V, int R, RowBlocks rb,
+__global__ void __launch_bounds__(256) ds_inplace_f32_kernel(float* __restrict__ S, int V, int R, RowPack rb,
                                                              int blk_off, const int32_t* __restrict__ ids,
                                                              const float* __restrict__ lse,
                                                              const float* __restrict__ g) {
@@ -478,20 +485,20 @@ __global__ void __launch_bounds__(256) ds_inplace_f32_kernel(float* __restrict__
   const int id = ids[n];
   for (int v = threadIdx.x; v < V; v += 256) row[v] = gn * ((v == id ? 1.f : 0.f) - expf(row[v] - L));
 }
-void launch_ds_inplace_f32(float* S, int V, int R, RowBlocks rb, int blk_off, const int32_t* ids, const float* lse,
+void launch_ds_inplace_f32(float* S, int V, int R, RowPack rb, int blk_off, const int32_t* ids, const float* lse,
                            const float* g, cudaStream_t s) {
   ds_inplace_f32_kernel<<<R, 256, 0, s>>>(S, V, R, rb, blk_off, ids, lse, g);
   note_launch();
 }
 
 __global__ void scatter_rows_f32_kernel(const float* __restrict__ dHp, float* __restrict__ dHidden, int H, int R,
-                                        RowBlocks rb, int blk_off) {
+                                        RowPack rb, int blk_off) {
   const int r = blockIdx.x;
   const long n = scratch_row_to_global(rb, blk_off, r);
   if (n < 0) return;
   for (int h = threadIdx.x; h < H; h += blockDim.x) dHidden[(size_t)n * H + h] = dHp[(size_t)r * H + h];
 }
-void launch_scatter_rows_f32(const float* dHp, float* dHidden, int H, int R, RowBlocks rb, int blk_off,
+void launch_scatter_rows_f32(const float* dHp, float* dHidden, int H, int R, RowPack rb, int blk_off,
                              cudaStream_t s) {
   scatter_rows_f32_kernel<<<R, 128, 0, s>>>(dHp, dHidden, H, R, rb, blk_off);
   note_launch();

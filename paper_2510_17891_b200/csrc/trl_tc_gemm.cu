@@ -43,7 +43,7 @@ constexpr long long WAIT_CYCLES = 4000000000LL;   // ~2-3 s at B200 clocks
 
 struct TcArgs {
   int N, K, m_blocks_fixed, blk_off, blk_cap, raster_band, rows_cap, V;
-  const int* nblk; const int* blk_row; const int* blk_n;
+  const int* nblk; const int* n_rows; const int* rowmap;
   const int32_t* ids; const float* lse; const float* g;
   float2* partials; float* tgt;
   __nv_bfloat16* dS; long ds_ld;
@@ -230,9 +230,9 @@ __device__ __forceinline__ void epilogue_tile(const TcArgs& p, uint32_t tmem_acc
   uint32_t v[32];
 
   if constexpr (EPI == TC_EPI_LSE) {
-    const int blk = p.blk_off + mb;
-    const bool valid = r < p.blk_n[blk];
-    const long grow = (long)p.blk_row[blk] + r;
+    const int prow_i = (p.blk_off + mb) * BM + r;          // packed row
+    const bool valid = prow_i < p.n_rows[0];
+    const long grow = valid ? (long)p.rowmap[prow_i] : 0;
     const int id = valid ? p.ids[grow] : -1;
     float m2 = -INFINITY, l = 0.f, tg = 0.f;
     bool has = false;
@@ -264,13 +264,13 @@ __device__ __forceinline__ void epilogue_tile(const TcArgs& p, uint32_t tmem_acc
         has = true;
       }
     }
-    const size_t prow = (size_t)blk * BM + r;
+    const size_t prow = (size_t)prow_i;
     p.partials[(size_t)nt * p.rows_cap + prow] = make_float2(m2 * LN2, l);
     if (has) p.tgt[prow] = tg;
   } else if constexpr (EPI == TC_EPI_DS) {
-    const int blk = p.blk_off + mb;
-    const bool valid = r < p.blk_n[blk];
-    const long grow = (long)p.blk_row[blk] + r;
+    const int prow_i = (p.blk_off + mb) * BM + r;          // packed row
+    const bool valid = prow_i < p.n_rows[0];
+    const long grow = valid ? (long)p.rowmap[prow_i] : 0;
     const int id = valid ? p.ids[grow] : -1;
     const float gg = valid ? p.g[grow] : 0.f;
     const float L2 = valid ? p.lse[grow] * LOG2E : 0.f;
@@ -297,9 +297,9 @@ __device__ __forceinline__ void epilogue_tile(const TcArgs& p, uint32_t tmem_acc
       wo.put<false>(w, n0 + c0, mb * BM + quad * 32);     // columns >= V are clipped by the TMA
     }
   } else if constexpr (EPI == TC_EPI_E) {
-    const int blk = p.blk_off + mb;
-    const bool valid = r < p.blk_n[blk];
-    const long grow = (long)p.blk_row[blk] + r;
+    const int prow_i = (p.blk_off + mb) * BM + r;          // packed row
+    const bool valid = prow_i < p.n_rows[0];
+    const long grow = valid ? (long)p.rowmap[prow_i] : 0;
     const int id = valid ? p.ids[grow] : -1;
     const float C2 = valid ? p.lse[grow] * LOG2E : 0.f;      // p.lse holds the shift c here
     const size_t srow = (size_t)mb * BM + r;
@@ -336,9 +336,9 @@ __device__ __forceinline__ void epilogue_tile(const TcArgs& p, uint32_t tmem_acc
     p.psum[(size_t)nt * p.rows_cap + srow] = sum;
     if (has) p.tgt[srow] = tg;
   } else if constexpr (EPI == TC_EPI_DH) {
-    const int blk = p.blk_off + mb;
-    const bool valid = r < p.blk_n[blk];
-    const long grow = (long)p.blk_row[blk] + r;
+    const int prow_i = (p.blk_off + mb) * BM + r;          // packed row
+    const bool valid = prow_i < p.n_rows[0];
+    const long grow = valid ? (long)p.rowmap[prow_i] : 0;
     const float rs = p.row_scale ? p.row_scale[(size_t)mb * BM + r] : 1.0f;
     __nv_bfloat16* out = p.dHidden + (size_t)grow * p.dh_ld;
     for (int c0 = 0; c0 < BN; c0 += 32) {
@@ -436,8 +436,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   auto a_row_of = [&](int mb) {
-    // forward GEMMs read hidden at the row block's own rows; the gradient GEMMs read chunk scratch
-    return (EPI == TC_EPI_LSE || EPI == TC_EPI_DS || EPI == TC_EPI_E) ? p.blk_row[p.blk_off + mb] : mb * BM;
+    // forward GEMMs read the packed hidden rows of the block; the gradient GEMMs read chunk scratch
+    return (EPI == TC_EPI_LSE || EPI == TC_EPI_DS || EPI == TC_EPI_E) ? (p.blk_off + mb) * BM : mb * BM;
   };
 
   if (warp == 0) {
@@ -630,7 +630,7 @@ int tc_num_sms() {
 cudaError_t launch_tc_gemm(const TcGemm& g, cudaStream_t s) {
   CUtensorMap tmA, tmB;
   if (!make_tmap(&tmA, g.A, g.a_rows, g.K, g.a_ld, BM, a_is_mn(g.epi))) return cudaErrorInvalidValue;
-  if (!make_tmap(&tmB, g.B, g.b_rows, g.K, g.b_ld, BN, b_is_mn(g.epi))) return cudaErrorInvalidValue;
+  if (!make_tmap(&tmB, g.B, g.b_rows, g.b_k > 0 ? g.b_k : g.K, g.b_ld, BN, b_is_mn(g.epi))) return cudaErrorInvalidValue;
   CUtensorMap tmOut = tmA;      // unused by the LSE and DH epilogues
   if (g.epi == TC_EPI_DS || g.epi == TC_EPI_E) {
     if (!make_out_tmap(&tmOut, g.dS, g.N, (long)g.blk_cap * BM, g.ds_ld, false)) return cudaErrorInvalidValue;
@@ -640,7 +640,7 @@ cudaError_t launch_tc_gemm(const TcGemm& g, cudaStream_t s) {
   TcArgs a;
   a.N = g.N; a.K = g.K; a.m_blocks_fixed = g.m_blocks; a.blk_off = g.blk_off; a.blk_cap = g.blk_cap;
   a.raster_band = g.raster_band > 0 ? g.raster_band : 16; a.rows_cap = g.rows_cap; a.V = g.V;
-  a.nblk = g.rb.nblk; a.blk_row = g.rb.blk_row; a.blk_n = g.rb.blk_n;
+  a.nblk = g.rb.nblk; a.n_rows = g.rb.n_rows; a.rowmap = g.rb.rowmap;
   a.ids = g.ids; a.lse = g.lse; a.g = g.g; a.partials = g.partials; a.tgt = g.tgt;
   a.dS = g.dS; a.ds_ld = g.ds_ld;
   a.dHidden = g.dHidden; a.dh_ld = g.dh_ld; a.dW = g.dW; a.dw_ld = g.dw_ld; a.status = g.status;
