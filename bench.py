@@ -189,7 +189,7 @@ def main():
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     stream = torch.cuda.current_stream()
 
-    def step_fused(ev=None):
+    def step_fused(ev=None, batch=batch):
         """One pass: old-policy scoring, HRD advantages, fused policy scoring + loss + backward."""
         mark = (lambda: None) if ev is None else (lambda: ev.append(_rec()))
         mark()
@@ -204,7 +204,7 @@ def main():
                               hrd["adv"], hrd["seg"], P, G, T, 0.2, 0.2, 0.1, fused_out, bufs["ws_bwd"], status, stream)
         mark()
 
-    def step_four(ev=None):
+    def step_four(ev=None, batch=batch):
         """The five C-ABI calls of one pass.  `ev` collects CUDA events around each call."""
         mark = (lambda: None) if ev is None else (lambda: ev.append(_rec()))
         mark()
@@ -264,26 +264,47 @@ def main():
              ["token_logprobs_policy", "token_logprobs_old", "hrd_advantages", "pg_loss_fwd", "pg_loss_bwd"])
     call_ms = {n: statistics.mean(ev[i].elapsed_time(ev[i + 1]) for ev in call_events) for i, n in enumerate(names)}
 
-    # ---- end-to-end: host buffers in, loss out, copies inside the timed region
-    host = {k: batch[k].cpu().pin_memory() for k in ("hidden", "hidden_old", "ids", "lens", "bnd", "r_plan", "r_code")}
+    # ---- end-to-end: host buffers in, loss out, copies inside the timed region.  Every step's
+    # inputs (both models' hidden states, ids, len, bnd, rewards) come from pinned host memory
+    # and its loss + statistics go back to the host; the upload of step i+1 runs on a copy
+    # stream into a second set of device buffers while step i computes (what a trainer does).
+    in_keys = ("hidden", "hidden_old", "ids", "lens", "bnd", "r_plan", "r_code")
+    host = {k: batch[k].cpu().pin_memory() for k in in_keys}
     host_out = torch.empty(5, dtype=torch.float32).pin_memory()
     h2d = sum(v.numel() * v.element_size() for v in host.values())
     d2h = host_out.numel() * 4
     e2e_steps = max(2, min(args.steps, 4))
+    sets = [batch, {**batch, **{k: torch.empty_like(batch[k]) for k in in_keys}}]
+    copy_stream = torch.cuda.Stream()
+    uploaded = [torch.cuda.Event(), torch.cuda.Event()]
+    consumed = [torch.cuda.Event(), torch.cuda.Event()]
 
-    def e2e_step():
-        for k, v in host.items():
-            batch[k].copy_(v, non_blocking=True)
-        step()
-        host_out[:1].copy_(bufs["loss"], non_blocking=True)
-        host_out[1:].copy_(bufs["stats"], non_blocking=True)
-        torch.cuda.synchronize()
+    def upload(i):
+        with torch.cuda.stream(copy_stream):
+            copy_stream.wait_event(consumed[i % 2])        # the step that last read this set has finished
+            for k, v in host.items():
+                sets[i % 2][k].copy_(v, non_blocking=True)
+            uploaded[i % 2].record(copy_stream)
 
-    e2e_step()
+    def e2e_run(n):
+        for e in consumed:
+            e.record(stream)
+        upload(0)
+        for i in range(n):
+            if i + 1 < n:
+                upload(i + 1)
+            stream.wait_event(uploaded[i % 2])
+            step(None, sets[i % 2])
+            consumed[i % 2].record(stream)
+            host_out[:1].copy_(bufs["loss"], non_blocking=True)
+            host_out[1:].copy_(bufs["stats"], non_blocking=True)
+            stream.synchronize()                           # the step's result is on the host
+
+    e2e_run(2)
     barrier()
     t0 = time.perf_counter()
-    for _ in range(e2e_steps):
-        e2e_step()
+    e2e_run(e2e_steps)
+    torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
     e2e_value, _, _ = dp.aggregate_throughput(1e3 * e2e_s, n_valid, e2e_steps, dev)
 
@@ -305,9 +326,9 @@ def main():
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        v_cpu, tok, sec, threads = oracle_sample_throughput(w, 2, 24)
+        v_cpu, tok, sec, threads = oracle_sample_throughput(w, 8, 48)
         cpu_baseline = dict(value=v_cpu, unit=UNIT, cores=threads, kind="oracle",
-                            sample=f"2 rollouts x T=24 ({tok} valid tokens, {sec:.1f} s), full H={H} V={V}, whole path in numpy fp64")
+                            sample=f"8 rollouts x T=48 ({tok} valid tokens, {sec:.1f} s), full H={H} V={V}, whole path in numpy fp64")
 
     if rank == 0:
         line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=max(args.warmup, 3),
