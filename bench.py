@@ -26,6 +26,10 @@ sys.path.insert(0, ROOT)
 METRIC = "scored_rollout_tokens_per_sec_fwd_bwd"
 UNIT = "tokens/s"
 WORKLOAD_ID = 2          # 8B-scale fwd+bwd: 8 prompts x 8 rollouts, T=2048, H=4096, V=151,936
+# DRAM bytes (read + write) of one tc_gemm_kernel<LSE> launch at WORKLOAD_ID, from the ncu capture of
+# the same kernel on the profile_small workload (0.897 GB: packed hidden once + W once per raster
+# band of 32 row blocks), scaled by (bands x bytes of W): see profiles/tc_gemm_profile_small_ncu_full.md
+LSE_TRAFFIC_BYTES = 2.85e10
 
 
 def load_peaks():
@@ -316,7 +320,8 @@ def main():
     achieved = flops_fwd / (t_fwd_ms * 1e-3) / 1e12
     peak = peaks["bf16_sustained"]
     roofline = dict(bound="tensor", kernel="tc_gemm_kernel<LSE> (inside trl_token_logprobs)", achieved=achieved,
-                    peak=peak, unit="TFLOP/s", frac=achieved / peak, traffic=None,
+                    peak=peak, unit="TFLOP/s", frac=achieved / peak,
+                    traffic=LSE_TRAFFIC_BYTES if args.workload == WORKLOAD_ID else None,
                     peak_source=f"{peaks['source']} sustained cuBLAS bf16")
     if args.path == "fused":     # policy forward + two gradient GEMMs = the metric's 6HV per token
         rest_alg = 6.0 * H * V * n_valid / (call_ms["pg_step_fused"] * 1e-3) / 1e12
