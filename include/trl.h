@@ -17,7 +17,7 @@
  *
  * Conventions.
  *  - Every pointer is a DEVICE pointer owned by the caller unless a comment says "host".
- *    The library allocates no device memory and keeps no state between calls; scratch
+ *    The library allocates no device memory and keeps no state that affects results; scratch
  *    comes from a caller-provided workspace of at least trl_workspace_bytes(...) bytes,
  *    256-byte aligned.  Workspaces may be reused between calls on the same stream.
  *  - All work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = default
@@ -70,6 +70,11 @@ typedef struct {
   float eps_lo;   /* lower clip: ratio clipped at 1 - eps_lo */
   float eps_hi;   /* upper clip: ratio clipped at 1 + eps_hi */
   float alpha;    /* weight of J^plan; J^code has weight 1   */
+  int clip_form;  /* 0: min[A s, A clip(s)], the HRD objective of Section 2.3.
+                     1: A min{s, clip(s)}, the form printed in the uniform-reward appendix; it
+                        differs for A < 0 (there s > 1+eps_hi saturates and s < 1-eps_lo does not) */
+  int agg_mode;   /* 0: (1/P) sum_i (1/G) sum_j (1/|o_ij|) sum_t, as in the paper.
+                     1: mean over all valid tokens of the call (not in the paper)              */
 } trl_pg_config;
 
 /* Bytes of workspace the given call wants for these shapes (recommended size).
@@ -127,6 +132,10 @@ int trl_hrd_advantages(const float* r_plan, const float* r_code,
  *   s = exp(logp - old_logp);  u = min(adv*s, adv*clip(s, 1-eps_lo, 1+eps_hi))
  *   loss = -(1/P) sum_i (1/G) sum_j (1/len_ij) sum_{t<len_ij} w_t u_t,  w = alpha (plan), 1 (code)
  *   g[n] = d loss / d logp[n] = -w adv s / (P G len) where the unclipped branch is the min, else 0
+ *
+ * cfg.clip_form / cfg.agg_mode select the two documented variants.  Uniform-reward GRPO (the
+ * paper's baseline, one advantage for all tokens of a rollout) is this call with
+ * r_plan = r_code = beta R^correct + (1 - beta) R^speedup in trl_hrd_advantages and alpha = 1.
  *
  * Both classes are divided by the whole response length |o_ij| = len.  The sum is taken in
  * a fixed order (bit-reproducible).

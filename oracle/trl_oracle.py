@@ -116,7 +116,8 @@ def hrd_advantages(r_plan, r_code, lens, bnd, P, G, T, adv_mode=0):
                 n_valid=int(lens.sum()))
 
 
-def pg_loss_fwd(logp, old_logp, adv, seg, lens, P, G, T, eps_lo=0.2, eps_hi=0.2, alpha=0.1):
+def pg_loss_fwd(logp, old_logp, adv, seg, lens, P, G, T, eps_lo=0.2, eps_hi=0.2, alpha=0.1, clip_form=0,
+                agg_mode=0):
     """Clipped importance-ratio surrogate with the plan/code weighting, and d loss / d logp.
 
     J = (1/P) sum_i [ alpha J^plan_i + J^code_i ],
@@ -128,6 +129,11 @@ def pg_loss_fwd(logp, old_logp, adv, seg, lens, P, G, T, eps_lo=0.2, eps_hi=0.2,
 
     g[n] = d loss / d logp[n] = -w A s / (P G len_b) when the unclipped branch is the
     minimum (A s <= A clip(s)), else 0; w = alpha for plan tokens, 1 for code tokens.
+
+    clip_form 1 replaces the min by A * min{s, clip(s, 1-eps, 1+eps)}, the form printed in the
+    appendix on uniform reward assignment (it differs from the above for A < 0).
+    agg_mode 1 replaces the (1/P)(1/G)(1/|o|) weights by one mean over all valid tokens of the
+    call (not in the paper).
 
     stats = [fraction of valid tokens with s > 1+eps_hi, fraction with s < 1-eps_lo,
              mean s over valid tokens, number of valid tokens].
@@ -147,6 +153,7 @@ def pg_loss_fwd(logp, old_logp, adv, seg, lens, P, G, T, eps_lo=0.2, eps_hi=0.2,
     n_hi = n_lo = 0
     sum_s = 0.0
     n_tok = 0
+    n_total = int(np.clip(lens, 0, T).sum())
     for i in range(P):
         Ji = 0.0
         for j in range(G):
@@ -159,17 +166,22 @@ def pg_loss_fwd(logp, old_logp, adv, seg, lens, P, G, T, eps_lo=0.2, eps_hi=0.2,
             A = adv[rows]
             w = np.where(seg[rows] == SEG_PLAN, alpha, np.where(seg[rows] == SEG_CODE, 1.0, 0.0))
             unclipped = A * s
-            clipped = A * np.clip(s, 1.0 - eps_lo, 1.0 + eps_hi)
-            u = np.minimum(unclipped, clipped)
-            Ji += (w * u).sum() / L
-            active = unclipped <= clipped
-            g[rows] = np.where(active, -w * A * s / (P * G * L), 0.0)
+            if clip_form == 0:
+                clipped = A * np.clip(s, 1.0 - eps_lo, 1.0 + eps_hi)
+                u = np.minimum(unclipped, clipped)
+                active = unclipped <= clipped
+            else:
+                u = A * np.minimum(s, np.clip(s, 1.0 - eps_lo, 1.0 + eps_hi))
+                active = s <= 1.0 + eps_hi
+            norm = (P * G * L) if agg_mode == 0 else n_total
+            Ji += (w * u).sum() / (L if agg_mode == 0 else 1.0)
+            g[rows] = np.where(active, -w * A * s / norm, 0.0)
             n_hi += int((s > 1.0 + eps_hi).sum())
             n_lo += int((s < 1.0 - eps_lo).sum())
             sum_s += float(s.sum())
             n_tok += L
-        J += Ji / G
-    J /= P
+        J += Ji / (G if agg_mode == 0 else 1.0)
+    J /= (P if agg_mode == 0 else max(n_total, 1))
     stats = np.array([n_hi / max(n_tok, 1), n_lo / max(n_tok, 1), sum_s / max(n_tok, 1), float(n_tok)])
     return -J, g, stats
 
@@ -222,14 +234,15 @@ def row_dhidden(hidden_row, W, tok, g_n):
 
 
 def full_step(hidden, W, hidden_old, W_old, ids, lens, bnd, r_plan, r_code, P, G, T,
-              eps_lo=0.2, eps_hi=0.2, alpha=0.1, adv_mode=0, old_logp=None):
+              eps_lo=0.2, eps_hi=0.2, alpha=0.1, adv_mode=0, old_logp=None, clip_form=0, agg_mode=0):
     """One pass of the whole path: score under pi_theta and pi_theta_old, HRD advantages,
     surrogate loss, backward.  If `old_logp` is given it replaces the pi_theta_old scoring."""
     logp, lse = token_logprobs(hidden, W, ids, lens, T)
     if old_logp is None:
         old_logp, _ = token_logprobs(hidden_old, W_old, ids, lens, T)
     hrd = hrd_advantages(r_plan, r_code, lens, bnd, P, G, T, adv_mode)
-    loss, g, stats = pg_loss_fwd(logp, old_logp, hrd["adv"], hrd["seg"], lens, P, G, T, eps_lo, eps_hi, alpha)
+    loss, g, stats = pg_loss_fwd(logp, old_logp, hrd["adv"], hrd["seg"], lens, P, G, T, eps_lo, eps_hi, alpha,
+                                 clip_form, agg_mode)
     dHidden, dW = pg_loss_bwd(hidden, W, ids, lens, lse, g, T)
     return dict(logp=logp, lse=lse, old_logp=old_logp, loss=loss, g=g, stats=stats,
                 dHidden=dHidden, dW=dW, **hrd)

@@ -19,7 +19,8 @@ class TrlError(RuntimeError):
 
 class PgConfig(ctypes.Structure):
     """trl_pg_config: clip range and plan weight (paper: eps = 0.2, alpha = 0.1)."""
-    _fields_ = [("eps_lo", ctypes.c_float), ("eps_hi", ctypes.c_float), ("alpha", ctypes.c_float)]
+    _fields_ = [("eps_lo", ctypes.c_float), ("eps_hi", ctypes.c_float), ("alpha", ctypes.c_float),
+                ("clip_form", ctypes.c_int), ("agg_mode", ctypes.c_int)]
 
 
 def lib_path():
@@ -157,7 +158,7 @@ def trl_hrd_advantages(r_plan, r_code, lens, bnd, P, G, T, adv_mode=0, out=None,
 
 
 def trl_pg_loss_fwd(logp, old_logp, adv, seg, lens, P, G, T, eps_lo=0.2, eps_hi=0.2, alpha=0.1,
-                    loss=None, g=None, stats=None, workspace=None, status=None, stream=None):
+                    loss=None, g=None, stats=None, workspace=None, status=None, stream=None, clip_form=0, agg_mode=0):
     """Clipped surrogate loss, d loss/d logp and clip statistics.  Returns (loss, g, stats)."""
     _dev(logp, old_logp, adv, seg, lens, loss, g, stats, workspace, status)
     dev = logp.device
@@ -170,22 +171,22 @@ def trl_pg_loss_fwd(logp, old_logp, adv, seg, lens, P, G, T, eps_lo=0.2, eps_hi=
     if workspace is None:
         workspace = _workspace(trl_workspace_bytes(TRL_CALL_PG_LOSS_FWD, P * G, T, 1, 1, TRL_F32), dev)
     rc = load_library().trl_pg_loss_fwd(_ptr(logp), _ptr(old_logp), _ptr(adv), _ptr(seg), _ptr(lens), P, G, T,
-                                        PgConfig(eps_lo, eps_hi, alpha), _ptr(loss), _ptr(g), _ptr(stats),
-                                        _ptr(workspace), workspace.numel(), _ptr(status), _stream(stream))
+                                        PgConfig(eps_lo, eps_hi, alpha, clip_form, agg_mode), _ptr(loss), _ptr(g),
+                                        _ptr(stats), _ptr(workspace), workspace.numel(), _ptr(status), _stream(stream))
     _check(rc, "trl_pg_loss_fwd")
     return loss, g, stats
 
 
 def trl_pg_loss_fwd_static(logp, old_logp, adv, seg, lens, P, G, T, loss, g, stats, eps_lo=0.2, eps_hi=0.2,
-                           alpha=0.1, status=None, stream=None):
+                           alpha=0.1, status=None, stream=None, clip_form=0, agg_mode=0):
     """trl_pg_loss_fwd for callers that cannot allocate: the scratch is a fixed array inside the
     library, and this wrapper allocates nothing either, so `loss` [1], `g` [P*G*T] and `stats`
     [4] (or None) must be passed in.  Limit P*G*ceil(T/4096) <= 65536.  Calls that may overlap
     on the GPU must not share a device.  Returns (loss, g, stats)."""
     _dev(logp, old_logp, adv, seg, lens, loss, g, stats, status)
     rc = load_library().trl_pg_loss_fwd_static(_ptr(logp), _ptr(old_logp), _ptr(adv), _ptr(seg), _ptr(lens), P, G, T,
-                                               PgConfig(eps_lo, eps_hi, alpha), _ptr(loss), _ptr(g), _ptr(stats),
-                                               _ptr(status), _stream(stream))
+                                               PgConfig(eps_lo, eps_hi, alpha, clip_form, agg_mode), _ptr(loss), _ptr(g),
+                                               _ptr(stats), _ptr(status), _stream(stream))
     _check(rc, "trl_pg_loss_fwd_static")
     return loss, g, stats
 
@@ -211,7 +212,7 @@ def trl_pg_loss_bwd(hidden, W, ids, lens, lse, g, T, dHidden=None, dW=None, work
 
 
 def trl_pg_step_fused(hidden, W, ids, lens, old_logp, lse_hint, adv, seg, P, G, T, eps_lo=0.2, eps_hi=0.2, alpha=0.1,
-                      out=None, workspace=None, status=None, stream=None):
+                      out=None, workspace=None, status=None, stream=None, clip_form=0, agg_mode=0):
     """Fused policy scoring + surrogate loss + backward (see include/trl.h).  `lse_hint` may be
     None.  Returns a dict with logp, lse, loss, g, stats, dHidden, dW."""
     _dev(hidden, W, ids, lens, old_logp, lse_hint, adv, seg, workspace, status)
@@ -231,7 +232,8 @@ def trl_pg_step_fused(hidden, W, ids, lens, old_logp, lse_hint, adv, seg, P, G, 
     if workspace is None:
         workspace = _workspace(trl_workspace_bytes(TRL_CALL_PG_STEP_FUSED, B, T, H, V, dt), dev)
     rc = load_library().trl_pg_step_fused(_ptr(hidden), _ptr(W), _ptr(ids), _ptr(lens), _ptr(old_logp), _ptr(lse_hint),
-                                          _ptr(adv), _ptr(seg), P, G, T, H, V, dt, PgConfig(eps_lo, eps_hi, alpha),
+                                          _ptr(adv), _ptr(seg), P, G, T, H, V, dt,
+                                          PgConfig(eps_lo, eps_hi, alpha, clip_form, agg_mode),
                                           _ptr(o["logp"]), _ptr(o["lse"]), _ptr(o["loss"]), _ptr(o["g"]),
                                           _ptr(o["stats"]), _ptr(o["dHidden"]), _ptr(o["dW"]), _ptr(workspace),
                                           workspace.numel(), _ptr(status), _stream(stream))
@@ -240,7 +242,7 @@ def trl_pg_step_fused(hidden, W, ids, lens, old_logp, lse_hint, adv, seg, P, G, 
 
 
 def hrd_pg_step(batch, P, G, T, eps_lo=0.2, eps_hi=0.2, alpha=0.1, adv_mode=0, old_logp=None, bufs=None,
-                status=None, stream=None, fused=False, use_hint=True):
+                status=None, stream=None, fused=False, use_hint=True, clip_form=0, agg_mode=0):
     """One pass of the whole path by calling the five C entry points in order: score under the
     current and the old policy, HRD advantages, surrogate loss, backward.  `bufs` may carry
     preallocated outputs / workspaces (keys as returned).  No arithmetic happens here."""
@@ -255,7 +257,7 @@ def hrd_pg_step(batch, P, G, T, eps_lo=0.2, eps_hi=0.2, alpha=0.1, adv_mode=0, o
                                  bufs.get("hrd"), status, stream)
         o = trl_pg_step_fused(batch["hidden"], batch["W"], batch["ids"], batch["lens"], old_logp,
                               old_lse if use_hint else None, hrd["adv"], hrd["seg"], P, G, T, eps_lo, eps_hi, alpha,
-                              bufs.get("fused_out"), bufs.get("ws_fused"), status, stream)
+                              bufs.get("fused_out"), bufs.get("ws_fused"), status, stream, clip_form, agg_mode)
         return dict(old_logp=old_logp, hrd=hrd, **o)
     logp, lse = trl_token_logprobs(batch["hidden"], batch["W"], batch["ids"], batch["lens"], T,
                                    bufs.get("logp"), bufs.get("lse"), bufs.get("ws_fwd"), status, stream)
@@ -266,7 +268,7 @@ def hrd_pg_step(batch, P, G, T, eps_lo=0.2, eps_hi=0.2, alpha=0.1, adv_mode=0, o
                              bufs.get("hrd"), status, stream)
     loss, g, stats = trl_pg_loss_fwd(logp, old_logp, hrd["adv"], hrd["seg"], batch["lens"], P, G, T, eps_lo, eps_hi,
                                      alpha, bufs.get("loss"), bufs.get("g"), bufs.get("stats"), bufs.get("ws_loss"),
-                                     status, stream)
+                                     status, stream, clip_form, agg_mode)
     dHidden, dW = trl_pg_loss_bwd(batch["hidden"], batch["W"], batch["ids"], batch["lens"], lse, g, T,
                                   bufs.get("dHidden"), bufs.get("dW"), bufs.get("ws_bwd"), status, stream)
     return dict(logp=logp, lse=lse, old_logp=old_logp, hrd=hrd, loss=loss, g=g, stats=stats, dHidden=dHidden, dW=dW)

@@ -10,6 +10,7 @@ namespace {
 constexpr int kRecommendedChunkRowsBf16 = 32768;
 constexpr int kRecommendedChunkRowsF32 = 2048;
 constexpr int kRasterBandFwd = 32;
+constexpr int kRasterBandFwdE = 24;   // forward tiles that also store E / dS
 constexpr int kRasterBandBwd = 4;
 
 int check_device() {
@@ -206,7 +207,8 @@ int trl_pg_loss_fwd(const float* logp, const float* old_logp, const float* adv, 
   (void)status_dev;
   if (!logp || !old_logp || !adv || !seg || !len || !loss || !g || !workspace) return TRL_ERR_INVALID_ARG;
   if (P <= 0 || G <= 0 || T <= 0 || (long)P * G > 65535 || (long)P * G * T >= (1L << 31)) return TRL_ERR_SHAPE;
-  if (!(cfg.eps_lo >= 0.f) || !(cfg.eps_hi >= 0.f) || !(cfg.alpha >= 0.f)) return TRL_ERR_INVALID_ARG;
+  if (!(cfg.eps_lo >= 0.f) || !(cfg.eps_hi >= 0.f) || !(cfg.alpha >= 0.f) || (cfg.clip_form & ~1) || (cfg.agg_mode & ~1))
+    return TRL_ERR_INVALID_ARG;
   if (workspace_bytes < trl_workspace_bytes(TRL_CALL_PG_LOSS_FWD, P * G, T, 1, 1, TRL_F32)) return TRL_ERR_WORKSPACE_TOO_SMALL;
   if (int e = check_device()) return e;
   launch_pg_loss(logp, old_logp, adv, seg, len, P, G, T, cfg, loss, g, stats, (float*)workspace, (cudaStream_t)stream);
@@ -249,7 +251,7 @@ int trl_pg_loss_bwd(const void* hidden, const void* W, const int32_t* ids, const
       a.rb = rb; a.blk_off = blk_off; a.blk_cap = CB; a.status = status_dev;
       // dS chunk = g (onehot - softmax), from a recomputed logits tile
       TcGemm ds = a;
-      ds.epi = TC_EPI_DS; ds.raster_band = kRasterBandFwd;
+      ds.epi = TC_EPI_DS; ds.raster_band = kRasterBandFwdE;
       ds.A = Xp; ds.a_rows = cap_rows; ds.a_ld = H; ds.B = W; ds.b_rows = V; ds.b_ld = H; ds.K = H; ds.N = V;
       ds.ids = ids; ds.lse = lse; ds.g = g; ds.dS = dS; ds.ds_ld = V;
       TRL_CUDA_OK(launch_tc_gemm(ds, s));
@@ -308,7 +310,8 @@ int trl_pg_step_fused(const void* hidden, const void* W, const int32_t* ids, con
   const int B = P * G;
   if (!shapes_ok(B, T, H, V)) return TRL_ERR_SHAPE;
   if (dt == TRL_BF16 && ((H % 8) || (V % 8))) return TRL_ERR_SHAPE;
-  if (!(cfg.eps_lo >= 0.f) || !(cfg.eps_hi >= 0.f) || !(cfg.alpha >= 0.f)) return TRL_ERR_INVALID_ARG;
+  if (!(cfg.eps_lo >= 0.f) || !(cfg.eps_hi >= 0.f) || !(cfg.alpha >= 0.f) || (cfg.clip_form & ~1) || (cfg.agg_mode & ~1))
+    return TRL_ERR_INVALID_ARG;
   if (((uintptr_t)workspace & 255) != 0) return TRL_ERR_INVALID_ARG;
   if (workspace_bytes < trl_workspace_bytes_min(TRL_CALL_PG_STEP_FUSED, B, T, H, V, dt)) return TRL_ERR_WORKSPACE_TOO_SMALL;
   if (int e = check_device()) return e;
@@ -370,7 +373,7 @@ int trl_pg_step_fused(const void* hidden, const void* W, const int32_t* ids, con
     a.blk_off = blk_off; a.blk_cap = CB;
     // forward tile -> E = exp(z - c), row sums, sampled token's logit
     TcGemm e = a;
-    e.epi = TC_EPI_E; e.raster_band = kRasterBandFwd;
+    e.epi = TC_EPI_E; e.raster_band = kRasterBandFwdE;
     e.A = Xp; e.a_rows = cap_rows; e.a_ld = H; e.B = W; e.b_rows = V; e.b_ld = H; e.K = H; e.N = V;
     e.ids = ids; e.lse = hint; e.dS = E; e.ds_ld = V; e.psum = psum; e.tgt = tgt; e.rows_cap = R;
     TRL_CUDA_OK(launch_tc_gemm(e, s));

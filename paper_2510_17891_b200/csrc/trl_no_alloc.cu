@@ -45,7 +45,8 @@ extern "C" int trl_pg_loss_fwd_static(const float* logp, const float* old_logp, 
   (void)status_dev;
   if (!logp || !old_logp || !adv || !seg || !len || !loss || !g) return TRL_ERR_INVALID_ARG;
   if (P <= 0 || G <= 0 || T <= 0 || (long)P * G > 65535 || (long)P * G * T >= (1L << 31)) return TRL_ERR_SHAPE;
-  if (!(cfg.eps_lo >= 0.f) || !(cfg.eps_hi >= 0.f) || !(cfg.alpha >= 0.f)) return TRL_ERR_INVALID_ARG;
+  if (!(cfg.eps_lo >= 0.f) || !(cfg.eps_hi >= 0.f) || !(cfg.alpha >= 0.f) || (cfg.clip_form & ~1) || (cfg.agg_mode & ~1))
+    return TRL_ERR_INVALID_ARG;
   // size limit of the built-in scratch: P*G*ceil(T/4096) slots
   if ((long)P * G * trl::pg_loss_tiles(T) > kStaticLossSlots) return TRL_ERR_WORKSPACE_TOO_SMALL;
   int major = 0, dev = 0;

@@ -189,6 +189,41 @@ void launch_hrd_advantages(const float* r_plan, const float* r_code, const int32
 constexpr int kLossTile = 4096;
 int pg_loss_tiles(int T) { return cdiv(T, kLossTile); }
 
+// One token of the surrogate: returns w*u and writes s and g (before the 1/normaliser factor
+// `inv` is applied to g by the caller's choice of inv).  Shared by the stand-alone loss kernel and
+// the fused step so both take the same decisions in the same arithmetic.
+struct TokenTerm { float wu, g, s; };
+__device__ __forceinline__ TokenTerm surrogate_token(float logp, float old_logp, float A, int sg,
+                                                    const trl_pg_config& cfg, float inv) {
+  const float lo = 1.0f - cfg.eps_lo, hi = 1.0f + cfg.eps_hi;
+  const float s = expf(logp - old_logp);
+  const float w = sg == 1 ? cfg.alpha : (sg == 2 ? 1.0f : 0.f);
+  const float unclipped = A * s;
+  TokenTerm t;
+  t.s = s;
+  if (cfg.clip_form == 0) {
+    const float clipped = A * fminf(fmaxf(s, lo), hi);
+    t.wu = w * fminf(unclipped, clipped);
+    t.g = (unclipped <= clipped) ? -w * A * s * inv : 0.f;
+  } else {                       // A * min{s, clip(s)} = A * min(s, 1 + eps_hi)
+    t.wu = w * A * fminf(s, hi);
+    t.g = (s <= hi) ? -w * A * s * inv : 0.f;
+  }
+  return t;
+}
+
+__device__ __forceinline__ long long total_valid_tokens(const int32_t* len, int B, int T, long long* sh) {
+  long long tot = 0;
+  for (int k = threadIdx.x; k < B; k += blockDim.x) tot += max(0, min(len[k], T));
+  for (int o = 16; o > 0; o >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, o);
+  if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = tot;
+  __syncthreads();
+  long long r = 0;
+  for (int k = 0; k < (int)(blockDim.x >> 5); ++k) r += sh[k];
+  __syncthreads();
+  return r;
+}
+
 __global__ void __launch_bounds__(256) pg_loss_stage1_kernel(
     const float* __restrict__ logp, const float* __restrict__ old_logp, const float* __restrict__ adv,
     const uint8_t* __restrict__ seg, const int32_t* __restrict__ len, int P, int G, int T, trl_pg_config cfg,
@@ -197,24 +232,24 @@ __global__ void __launch_bounds__(256) pg_loss_stage1_kernel(
   const int L = max(0, min(len[b], T));
   const int t_begin = blockIdx.x * kLossTile, t_end = min(T, t_begin + kLossTile);
   const size_t base = (size_t)b * T;
-  const float inv = L > 0 ? 1.0f / ((float)P * (float)G * (float)L) : 0.f;
+  __shared__ long long sh_tot[8];
+  float inv = L > 0 ? 1.0f / ((float)P * (float)G * (float)L) : 0.f;
+  if (cfg.agg_mode == 1) {
+    const long long ntok = total_valid_tokens(len, P * G, T, sh_tot);
+    inv = ntok > 0 ? 1.0f / (float)ntok : 0.f;
+  }
   const float lo = 1.0f - cfg.eps_lo, hi = 1.0f + cfg.eps_hi;
   float acc = 0.f, n_hi = 0.f, n_lo = 0.f, sum_s = 0.f;
   for (int t = t_begin + tid; t < t_end; t += 256) {
     float gn = 0.f;
     if (t < L) {
       const size_t n = base + t;
-      const float s = expf(logp[n] - old_logp[n]);
-      const float A = adv[n];
-      const int sg = seg[n];
-      const float w = sg == 1 ? cfg.alpha : (sg == 2 ? 1.0f : 0.f);
-      const float unclipped = A * s;
-      const float clipped = A * fminf(fmaxf(s, lo), hi);
-      acc += w * fminf(unclipped, clipped);
-      if (unclipped <= clipped) gn = -w * A * s * inv;
-      n_hi += s > hi ? 1.f : 0.f;
-      n_lo += s < lo ? 1.f : 0.f;
-      sum_s += s;
+      const TokenTerm tt = surrogate_token(logp[n], old_logp[n], adv[n], seg[n], cfg, inv);
+      acc += tt.wu;
+      gn = tt.g;
+      n_hi += tt.s > hi ? 1.f : 0.f;
+      n_lo += tt.s < lo ? 1.f : 0.f;
+      sum_s += tt.s;
     }
     g[base + t] = gn;
   }
@@ -235,7 +270,7 @@ __global__ void __launch_bounds__(256) pg_loss_stage1_kernel(
 
 __global__ void __launch_bounds__(256) pg_loss_stage2_kernel(const float* __restrict__ partials,
                                                              const int32_t* __restrict__ len, int P, int G, int T,
-                                                             int tiles, float* __restrict__ loss,
+                                                             int tiles, int agg_mode, float* __restrict__ loss,
                                                              float* __restrict__ stats) {
   __shared__ double red[4][256];
   const int tid = threadIdx.x, B = P * G;
@@ -247,7 +282,7 @@ __global__ void __launch_bounds__(256) pg_loss_stage2_kernel(const float* __rest
       const float* p = partials + ((size_t)b * tiles + k) * 4;
       a += p[0]; nh += p[1]; nl += p[2]; ss += p[3];
     }
-    if (L > 0) J += a / L;
+    if (L > 0) J += agg_mode == 1 ? a : a / L;
   }
   red[0][tid] = J; red[1][tid] = nh; red[2][tid] = nl; red[3][tid] = ss;
   __syncthreads();
@@ -257,7 +292,7 @@ __global__ void __launch_bounds__(256) pg_loss_stage2_kernel(const float* __rest
       for (int k = 0; k < 256; ++k) t[q] += red[q][k];
     long long ntok = 0;
     for (int b = 0; b < B; ++b) ntok += max(0, min(len[b], T));
-    loss[0] = (float)(-t[0] / ((double)P * (double)G));
+    loss[0] = agg_mode == 1 ? (float)(ntok > 0 ? -t[0] / (double)ntok : 0.0) : (float)(-t[0] / ((double)P * (double)G));
     if (stats) {
       const double d = ntok > 0 ? (double)ntok : 1.0;
       stats[0] = (float)(t[1] / d); stats[1] = (float)(t[2] / d); stats[2] = (float)(t[3] / d);
@@ -273,7 +308,7 @@ void launch_pg_loss(const float* logp, const float* old_logp, const float* adv, 
   dim3 grid(tiles, P * G);
   pg_loss_stage1_kernel<<<grid, 256, 0, s>>>(logp, old_logp, adv, seg, len, P, G, T, cfg, g, partials);
   note_launch();
-  pg_loss_stage2_kernel<<<1, 256, 0, s>>>(partials, len, P, G, T, tiles, loss, stats);
+  pg_loss_stage2_kernel<<<1, 256, 0, s>>>(partials, len, P, G, T, tiles, cfg.agg_mode, loss, stats);
   note_launch();
 }
 
@@ -387,14 +422,9 @@ __global__ void __launch_bounds__(128) fused_merge_kernel(FusedMergeArgs a) {
   a.logp[n] = lp;
   a.lse[n] = lse;
   const int L = max(0, min(a.len[b], a.T));
-  const float inv = 1.0f / ((float)a.P * (float)a.G * (float)L);
-  const float s = expf(lp - a.old_logp[n]);
-  const float A = a.adv[n];
-  const int sg = a.seg[n];
-  const float w = sg == 1 ? a.cfg.alpha : (sg == 2 ? 1.0f : 0.f);
-  const float unclipped = A * s;
-  const float clipped = A * fminf(fmaxf(s, 1.0f - a.cfg.eps_lo), 1.0f + a.cfg.eps_hi);
-  const float gn = (id_ok && unclipped <= clipped) ? -w * A * s * inv : 0.f;
+  const float inv = a.cfg.agg_mode == 1 ? 1.0f / (float)a.rb.n_rows[0] : 1.0f / ((float)a.P * (float)a.G * (float)L);
+  const TokenTerm tt = surrogate_token(lp, a.old_logp[n], a.adv[n], a.seg[n], a.cfg, inv);
+  const float gn = id_ok ? tt.g : 0.f;
   a.g[n] = gn;
   a.neg_alpha[r] = -gn * expf(c - lse);
   if (gn != 0.f) {

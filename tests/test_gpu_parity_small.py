@@ -20,7 +20,7 @@ def trl():
 
 
 def run_and_compare(trl, w, batch=None, explicit_old=False, alpha=0.1, eps=0.2, adv_mode=0, fused=False,
-                    use_hint=True):
+                    use_hint=True, clip_form=0, agg_mode=0):
     dev = "cuda:0"
     batch = synth.make_batch(w, device=dev) if batch is None else batch
     oi = oracle_inputs(batch)
@@ -31,10 +31,11 @@ def run_and_compare(trl, w, batch=None, explicit_old=False, alpha=0.1, eps=0.2, 
         old_logp_o = (lp + oi["old_noise"]).astype(np.float32).astype(np.float64)
         old_logp_g = torch.tensor(old_logp_o, dtype=torch.float32, device=dev)
     ref = orc.full_step(oi["hidden"], oi["W"], oi["hidden_old"], oi["W_old"], oi["ids"], oi["lens"], oi["bnd"],
-                        oi["r_plan"], oi["r_code"], w.P, w.G, w.T, eps, eps, alpha, adv_mode, old_logp=old_logp_o)
+                        oi["r_plan"], oi["r_code"], w.P, w.G, w.T, eps, eps, alpha, adv_mode, old_logp=old_logp_o,
+                        clip_form=clip_form, agg_mode=agg_mode)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     out = trl.hrd_pg_step(batch, w.P, w.G, w.T, eps, eps, alpha, adv_mode, old_logp=old_logp_g, status=status,
-                          fused=fused, use_hint=use_hint)
+                          fused=fused, use_hint=use_hint, clip_form=clip_form, agg_mode=agg_mode)
     torch.cuda.synchronize()
     trl.check_status(status)
     hrd = out["hrd"]
@@ -218,6 +219,36 @@ def test_fused_step_any_reasonable_hint_gives_same_result_and_bad_hint_is_flagge
     trl.trl_pg_step_fused(*args, old_lse - 500.0, hrd["adv"], hrd["seg"], w.P, w.G, w.T, status=status)
     torch.cuda.synchronize()
     assert int(status.item()) & (1 << 9)
+
+
+@pytest.mark.parametrize("fused", [False, True])
+def test_documented_loss_variants(trl, fused):
+    """Appendix clip form A*min{s, clip(s)} (uniform-reward GRPO as printed: one reward for both
+    classes, alpha = 1) and token-mean aggregation, against the oracle."""
+    w = synth.scaled(synth.CONFIGS[2], name="variants", P=2, G=4, T=200, H=256, V=1536, sigma_old=0.15)
+    batch = synth.make_batch(w, device="cuda:0")
+    run_and_compare(trl, w, batch=batch, fused=fused, clip_form=1)
+    run_and_compare(trl, w, batch=batch, fused=fused, agg_mode=1)
+    batch["r_code"] = batch["r_plan"] = 0.7 * batch["r_code"] + 0.3 * batch["r_plan"]     # beta = 0.7 mixture
+    run_and_compare(trl, w, batch=batch, fused=fused, clip_form=1, alpha=1.0)
+    run_and_compare(trl, synth.CONFIGS[0], fused=fused, clip_form=1, agg_mode=1)
+
+
+def test_fused_step_minimum_workspace_chunks(trl):
+    """One 128-row chunk at a time must give what one big chunk gives."""
+    w = synth.scaled(synth.CONFIGS[2], name="fused_chunks", P=1, G=3, T=300, H=128, V=520)
+    batch = synth.make_batch(w, device="cuda:0")
+    old_logp, old_lse = trl.trl_token_logprobs(batch["hidden_old"], batch["W_old"], batch["ids"], batch["lens"], w.T)
+    hrd = trl.trl_hrd_advantages(batch["r_plan"], batch["r_code"], batch["lens"], batch["bnd"], w.P, w.G, w.T)
+    args = (batch["hidden"], batch["W"], batch["ids"], batch["lens"], old_logp, old_lse, hrd["adv"], hrd["seg"], w.P, w.G, w.T)
+    ref = trl.trl_pg_step_fused(*args)
+    nmin = trl.trl_workspace_bytes_min(trl.TRL_CALL_PG_STEP_FUSED, w.B, w.T, w.H, w.V, trl.TRL_BF16)
+    assert nmin < trl.trl_workspace_bytes(trl.TRL_CALL_PG_STEP_FUSED, w.B, w.T, w.H, w.V, trl.TRL_BF16)
+    out = trl.trl_pg_step_fused(*args, workspace=torch.empty(nmin, dtype=torch.uint8, device="cuda:0"))
+    torch.cuda.synchronize()
+    assert torch.equal(out["logp"], ref["logp"]) and torch.equal(out["g"], ref["g"]) and torch.equal(out["dHidden"], ref["dHidden"])
+    assert float(out["loss"]) == float(ref["loss"])
+    assert rel_fro(f64(out["dW"]), f64(ref["dW"])) < 1e-5
 
 
 def test_minimum_workspace_gives_same_backward(trl):

@@ -367,3 +367,71 @@ def test_full_step_composes():
     old, _ = orc.token_logprobs(p["hidden"], Wo, p["ids"], p["lens"], p["T"])
     np.testing.assert_array_equal(out["old_logp"], old)
     assert np.isfinite(out["loss"]) and out["dW"].shape == p["W"].shape
+
+
+# ------------------------------------------------------------ documented variants of the loss
+
+@pytest.mark.parametrize("s,A,u,active", [
+    (1.5, 2.0, 2.0 * 1.2, False),     # same as the main form for A > 0
+    (0.5, 2.0, 2.0 * 0.5, True),
+    (1.5, -2.0, -2.0 * 1.2, False),   # A < 0: s above 1+eps saturates (unlike the main form)
+    (0.5, -2.0, -2.0 * 0.5, True),    # A < 0: s below 1-eps does not saturate (unlike the main form)
+])
+def test_appendix_clip_form_single_token(s, A, u, active):
+    loss, g, _ = orc.pg_loss_fwd(np.array([math.log(s) - 1.0]), np.array([-1.0]), np.array([A]),
+                                 np.array([2], dtype=np.uint8), np.array([1]), 1, 1, 1, 0.2, 0.2, 0.1, clip_form=1)
+    assert abs(loss + u) < 1e-14
+    assert abs(g[0] - (-A * s if active else 0.0)) < 1e-14
+
+
+def test_appendix_form_is_uniform_grpo_as_printed_and_fd_gradient():
+    # alpha = 1, r_plan = r_code, clip_form = 1: L_GRPO of the appendix, A * min{s, clip(s)}, by loops
+    p = _tiny_problem(31, P=2, G=4, T=8)
+    P, G, T = p["P"], p["G"], p["T"]
+    r = _rng(32)
+    old = -r.random(P * G * T) * 4
+    logp = old + r.standard_normal(P * G * T) * 0.3
+    hu = orc.hrd_advantages(p["r_plan"], p["r_plan"], p["lens"], p["bnd"], P, G, T)
+    lu, g, _ = orc.pg_loss_fwd(logp, old, hu["adv"], hu["seg"], p["lens"], P, G, T, 0.2, 0.2, 1.0, clip_form=1)
+    J = 0.0
+    for i in range(P):
+        mu = sum(p["r_plan"][i * G + j] for j in range(G)) / G
+        for j in range(G):
+            b = i * G + j
+            A = p["r_plan"][b] - mu
+            acc = sum(A * min(math.exp(logp[b * T + t] - old[b * T + t]),
+                              min(max(math.exp(logp[b * T + t] - old[b * T + t]), 0.8), 1.2))
+                      for t in range(p["lens"][b]))
+            J += acc / p["lens"][b] / G
+    assert abs(lu + J / P) < 1e-13
+    h = 1e-6
+    for n in range(0, logp.size, 5):
+        s = math.exp(logp[n] - old[n])
+        if abs(s - 1.2) < 1e-3:
+            continue
+        lp = logp.copy(); lm = logp.copy()
+        lp[n] += h; lm[n] -= h
+        fp = orc.pg_loss_fwd(lp, old, hu["adv"], hu["seg"], p["lens"], P, G, T, 0.2, 0.2, 1.0, clip_form=1)[0]
+        fm = orc.pg_loss_fwd(lm, old, hu["adv"], hu["seg"], p["lens"], P, G, T, 0.2, 0.2, 1.0, clip_form=1)[0]
+        assert abs((fp - fm) / (2 * h) - g[n]) < 1e-8
+
+
+def test_token_mean_aggregation_closed_form_and_fd():
+    p = _tiny_problem(33, P=3, G=4, T=9)
+    P, G, T = p["P"], p["G"], p["T"]
+    hrd = orc.hrd_advantages(p["r_plan"], p["r_code"], p["lens"], p["bnd"], P, G, T)
+    logp = -_rng(34).random(P * G * T) * 5
+    alpha = 0.37
+    loss, g, _ = orc.pg_loss_fwd(logp, logp.copy(), hrd["adv"], hrd["seg"], p["lens"], P, G, T, 0.2, 0.2, alpha, agg_mode=1)
+    # s = 1: loss = -sum_b [alpha A_plan n_plan + A_code n_code] / sum_b len
+    num = sum(alpha * hrd["A_plan"][b] * p["bnd"][b] + hrd["A_code"][b] * (p["lens"][b] - p["bnd"][b]) for b in range(P * G))
+    assert abs(loss + num / p["lens"].sum()) < 1e-13
+    h = 1e-6
+    old = logp - 0.05
+    _, g, _ = orc.pg_loss_fwd(logp, old, hrd["adv"], hrd["seg"], p["lens"], P, G, T, 0.2, 0.2, alpha, agg_mode=1)
+    for n in range(0, logp.size, 7):
+        lp = logp.copy(); lm = logp.copy()
+        lp[n] += h; lm[n] -= h
+        fp = orc.pg_loss_fwd(lp, old, hrd["adv"], hrd["seg"], p["lens"], P, G, T, 0.2, 0.2, alpha, agg_mode=1)[0]
+        fm = orc.pg_loss_fwd(lm, old, hrd["adv"], hrd["seg"], p["lens"], P, G, T, 0.2, 0.2, alpha, agg_mode=1)[0]
+        assert abs((fp - fm) / (2 * h) - g[n]) < 1e-8
