@@ -58,7 +58,7 @@ size_t loss_bytes(int B, int T) { return align_up((size_t)B * pg_loss_tiles(T) *
 size_t fused_fixed_bf16(int B, int T, int H, int V) { return bwd_fixed_bf16(B, T, H, V) + loss_bytes(B, T); }
 size_t fused_per_rows_bf16(int H, int V, int R) {
   return align_up((size_t)H * R * 2, 256) + align_up((size_t)R * V * 2, 256) + align_up((size_t)cdiv(V, 256) * R * 4, 256) +
-         2 * align_up((size_t)R * 4, 256);
+         2 * align_up((size_t)R * 4, 256) + align_up((size_t)(R / kRowBlock) * 4, 256);
 }
 
 // largest multiple of 128 rows (<= cap) whose scratch fits into `avail` bytes
@@ -343,6 +343,7 @@ int trl_pg_step_fused(const void* hidden, const void* W, const int32_t* ids, con
   float* psum = cv.take<float>((size_t)nt * R);
   float* tgt = cv.take<float>(R);
   float* neg_alpha = cv.take<float>(R);
+  int* blk_active = cv.take<int>(R / kRowBlock);
 
   launch_build_row_pack(len, B, T, rb, status_dev, s);
   TRL_CUDA_OK(cudaMemsetAsync(dW, 0, (size_t)V * H * sizeof(float), s));
@@ -378,20 +379,20 @@ int trl_pg_step_fused(const void* hidden, const void* W, const int32_t* ids, con
     e.ids = ids; e.lse = hint; e.dS = E; e.ds_ld = V; e.psum = psum; e.tgt = tgt; e.rows_cap = R;
     TRL_CUDA_OK(launch_tc_gemm(e, s));
     FusedMergeArgs m{psum, tgt, nt, R, rb, blk_off, ids, len, hint, old_logp, adv, seg, P, G, T, V, cfg,
-                     logp, lse, g, neg_alpha, E, status_dev};
+                     logp, lse, g, neg_alpha, blk_active, E, status_dev};
     launch_fused_merge(m, s);
     launch_pack_rows_bf16(Xp, Xs, H, R, rb, blk_off * kRowBlock, 1, neg_alpha, s);
     // dHidden rows = neg_alpha * (E' W)
     TcGemm dh = a;
     dh.epi = TC_EPI_DH; dh.raster_band = kRasterBandBwd;
     dh.A = E; dh.a_rows = R; dh.a_ld = V; dh.B = W; dh.b_rows = H; dh.b_ld = H; dh.K = V; dh.N = H;
-    dh.dHidden = (__nv_bfloat16*)dHidden; dh.dh_ld = H; dh.row_scale = neg_alpha;
+    dh.dHidden = (__nv_bfloat16*)dHidden; dh.dh_ld = H; dh.row_scale = neg_alpha; dh.blk_active = blk_active;
     TRL_CUDA_OK(launch_tc_gemm(dh, s));
     // dW += E'^T (neg_alpha * hidden)
     TcGemm dw = a;
     dw.epi = TC_EPI_DW; dw.raster_band = kRasterBandBwd;
     dw.A = E; dw.a_rows = V; dw.a_ld = V; dw.B = Xs; dw.b_rows = H; dw.b_ld = H; dw.K = R; dw.N = H;
-    dw.m_blocks = cdiv(V, kRowBlock); dw.dW = dW; dw.dw_ld = H; dw.V = V;
+    dw.m_blocks = cdiv(V, kRowBlock); dw.dW = dW; dw.dw_ld = H; dw.V = V; dw.blk_active = blk_active;
     TRL_CUDA_OK(launch_tc_gemm(dw, s));
   }
   // loss, statistics (and g once more, identically) over all rows now that logp is complete

@@ -57,6 +57,7 @@ struct FusedMergeArgs {
   const int32_t* ids; const int32_t* len; const float* hint; const float* old_logp; const float* adv;
   const uint8_t* seg; int P, G, T, V; trl_pg_config cfg;
   float* logp; float* lse; float* g; float* neg_alpha;
+  int* blk_active;                  // [R/128] 1 if any row of the block has a non-zero factor
   __nv_bfloat16* E;
   int32_t* status;
 };
@@ -107,6 +108,7 @@ struct TcGemm {
   float* dW; long dw_ld; int V;                        // DW
   float* psum;                                         // E: row sums per vocabulary tile [n_tiles, rows_cap]
   const float* row_scale;                              // DH: optional per-scratch-row factor
+  const int* blk_active;                               // DH, DW: optional per-row-block activity flags of the chunk
   int32_t* status;
 };
 // returns cudaSuccess or the error of tensor-map creation / launch

@@ -403,35 +403,40 @@ void launch_pack_rows_bf16(const __nv_bfloat16* src, __nv_bfloat16* out, int H, 
 // sampled token's entry of E.
 // ------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(128) fused_merge_kernel(FusedMergeArgs a) {
+  // one CTA = one 128-row block of the chunk
   const int r = blockIdx.x * 128 + threadIdx.x;
-  if (r >= a.R) return;
   const int q = a.blk_off * kRowBlock + r;
-  if (q >= a.rb.nblk[0] * kRowBlock) return;
-  if (q >= a.rb.n_rows[0]) { a.neg_alpha[r] = 0.f; return; }
-  const size_t n = (size_t)a.rb.rowmap[q];
-  const int b = (int)(n / a.T);
-  float sum = 0.f;
-  for (int k = 0; k < a.n_tiles; ++k) sum += a.psum[(size_t)k * a.R + r];
-  const float c = a.hint[n];
-  const float lse = c + logf(sum);
-  const int id = a.ids[n];
-  const bool id_ok = (unsigned)id < (unsigned)a.V;
-  if (!id_ok) flag_status(a.status, TRL_ERR_BAD_INDEX);
-  if (!(sum > 0.f) || !isfinite(sum)) flag_status(a.status, TRL_ERR_BAD_HINT);
-  const float lp = id_ok ? a.tgt[r] - lse : 0.f;
-  a.logp[n] = lp;
-  a.lse[n] = lse;
-  const int L = max(0, min(a.len[b], a.T));
-  const float inv = a.cfg.agg_mode == 1 ? 1.0f / (float)a.rb.n_rows[0] : 1.0f / ((float)a.P * (float)a.G * (float)L);
-  const TokenTerm tt = surrogate_token(lp, a.old_logp[n], a.adv[n], a.seg[n], a.cfg, inv);
-  const float gn = id_ok ? tt.g : 0.f;
-  a.g[n] = gn;
-  a.neg_alpha[r] = -gn * expf(c - lse);
-  if (gn != 0.f) {
-    const float beta = expf(lse - c);
-    __nv_bfloat16* e = a.E + (size_t)r * a.V + id;
-    *e = __float2bfloat16_rn(__bfloat162float(*e) - beta);
+  if (blockIdx.x * 128 >= a.R || a.blk_off + (int)blockIdx.x >= a.rb.nblk[0]) return;   // whole block not live
+  float gn = 0.f;
+  if (r < a.R && q < a.rb.n_rows[0]) {
+    const size_t n = (size_t)a.rb.rowmap[q];
+    const int b = (int)(n / a.T);
+    float sum = 0.f;
+    for (int k = 0; k < a.n_tiles; ++k) sum += a.psum[(size_t)k * a.R + r];
+    const float c = a.hint[n];
+    const float lse = c + logf(sum);
+    const int id = a.ids[n];
+    const bool id_ok = (unsigned)id < (unsigned)a.V;
+    if (!id_ok) flag_status(a.status, TRL_ERR_BAD_INDEX);
+    if (!(sum > 0.f) || !isfinite(sum)) flag_status(a.status, TRL_ERR_BAD_HINT);
+    const float lp = id_ok ? a.tgt[r] - lse : 0.f;
+    a.logp[n] = lp;
+    a.lse[n] = lse;
+    const int L = max(0, min(a.len[b], a.T));
+    const float inv = a.cfg.agg_mode == 1 ? 1.0f / (float)a.rb.n_rows[0] : 1.0f / ((float)a.P * (float)a.G * (float)L);
+    const TokenTerm tt = surrogate_token(lp, a.old_logp[n], a.adv[n], a.seg[n], a.cfg, inv);
+    gn = id_ok ? tt.g : 0.f;
+    a.g[n] = gn;
+    if (gn != 0.f) {
+      const float beta = expf(lse - c);
+      __nv_bfloat16* e = a.E + (size_t)r * a.V + id;
+      *e = __float2bfloat16_rn(__bfloat162float(*e) - beta);
+    }
+    gn = -gn * expf(c - lse);
   }
+  if (r < a.R) a.neg_alpha[r] = gn;
+  const int any = __syncthreads_or(gn != 0.f);
+  if (threadIdx.x == 0) a.blk_active[blockIdx.x] = any;
 }
 
 void launch_fused_merge(const FusedMergeArgs& a, cudaStream_t s) {

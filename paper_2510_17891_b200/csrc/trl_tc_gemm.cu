@@ -50,6 +50,7 @@ struct TcArgs {
   __nv_bfloat16* dHidden; long dh_ld;
   float* dW; long dw_ld;
   float* psum; const float* row_scale;
+  const int* blk_active;     // per row block of the chunk: 0 = every row has a zero gradient factor (may be null)
   int32_t* status;
 };
 
@@ -415,8 +416,23 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const int K = (EPI == TC_EPI_DW) ? live * BM : p.K;
   const int NT = (p.N + BN - 1) / BN;
   const int nkb = (K + BK - 1) / BK;
-  const int total = (nkb > 0) ? MS * NT : 0;
+  int total = (nkb > 0) ? MS * NT : 0;
+  if (EPI == TC_EPI_DW && p.blk_active) {       // row blocks whose rows all have a zero factor add nothing to dW
+    int n_act = 0;
+    for (int i = 0; i < live; ++i) n_act += p.blk_active[i] != 0;
+    if (n_act == 0) total = 0;
+  }
   if (total == 0 || (int)blockIdx.x >= total) return;
+  // Which M sub-blocks of a CTA tile take part (identical decision in every role): present, and for
+  // dHidden not marked inactive.  Which k-blocks take part: for dW, those of active row blocks.
+  auto tile_mask = [&](int ms) {
+    const int nm = min(MT, MB - ms * MT);
+    int m = 0;
+    for (int j = 0; j < nm; ++j)
+      if (!(EPI == TC_EPI_DH && p.blk_active) || p.blk_active[ms * MT + j] != 0) m |= 1 << j;
+    return m;
+  };
+  auto kb_on = [&](int kb) { return !(EPI == TC_EPI_DW && p.blk_active) || p.blk_active[kb >> 1] != 0; };
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
@@ -448,15 +464,17 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x) {
         int ms, nt;
         tile_coords(tile, MS, NT, p.raster_band, ms, nt);
-        const int nm = min(MT, MB - ms * MT);                 // M blocks present in this tile (1 or 2)
+        const int mask = tile_mask(ms);                        // M blocks of this tile that take part
+        if (mask == 0) continue;
         const int b_row = nt * BN;
         for (int kb = 0; kb < nkb; ++kb) {
+          if (!kb_on(kb)) continue;
           if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status))) break;
-          mbar_expect_tx(full_bar(stage), (uint32_t)(nm * A_BYTES + B_BYTES));
+          mbar_expect_tx(full_bar(stage), (uint32_t)(__popc(mask) * A_BYTES + B_BYTES));
           const uint32_t sa = smem_base + stage * STG;
 #pragma unroll
           for (int j = 0; j < MT; ++j) {
-            if (j < nm) {
+            if (mask & (1 << j)) {
               const int a_row = a_row_of(ms * MT + j);
               if constexpr (a_is_mn(EPI)) {       // two 64(M) x 64(K) boxes
                 tma_load_2d(sa + j * A_BYTES, &tmA, a_row, kb * BK, full_bar(stage));
@@ -491,11 +509,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x) {
         int ms, nt;
         tile_coords(tile, MS, NT, p.raster_band, ms, nt);
-        const int nm = min(MT, MB - ms * MT);
+        const int mask = tile_mask(ms);
+        if (mask == 0) continue;
         if (!(ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, p.status))) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * MT * BN);
+        bool first_kb = true;                                  // the first k-block that runs overwrites the accumulator
         for (int kb = 0; kb < nkb; ++kb) {
+          if (!kb_on(kb)) continue;
           if (!(ok = mbar_wait(full_bar(stage), phase, abort_flag, p.status))) break;
           tc_fence_after();
           const uint32_t sa = smem_base + stage * STG;
@@ -506,13 +527,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           constexpr uint64_t ka = a_is_mn(EPI) ? 128 : 2, kbs = b_is_mn(EPI) ? 128 : 2;
 #pragma unroll
           for (int j = 0; j < MT; ++j) {
-            if (j < nm) {
+            if (mask & (1 << j)) {
               const uint64_t da = a_is_mn(EPI) ? make_mnmajor_sw128_desc(sa + j * A_BYTES) : make_kmajor_sw128_desc(sa + j * A_BYTES);
 #pragma unroll
               for (int k = 0; k < BK / UMMA_K; ++k)
-                tc_mma_bf16(d_tmem + (uint32_t)(j * BN), da + ka * k, db + kbs * k, idesc, (uint32_t)((kb | k) != 0));
+                tc_mma_bf16(d_tmem + (uint32_t)(j * BN), da + ka * k, db + kbs * k, idesc, (uint32_t)(!(first_kb && k == 0)));
             }
           }
+          first_kb = false;
           tc_commit(empty_bar(stage));
           if (++stage == NSTAGE) { stage = 0; phase ^= 1u; }
         }
@@ -530,14 +552,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     for (int tile = blockIdx.x; tile < total; tile += gridDim.x) {
       int ms, nt;
       tile_coords(tile, MS, NT, p.raster_band, ms, nt);
-      const int nm = min(MT, MB - ms * MT);
+      const int mask = tile_mask(ms);
+      if (mask == 0) continue;
       bool ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.status);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
 #pragma unroll
       for (int j = 0; j < MT; ++j)
-        if (j < nm) epilogue_tile<EPI>(p, tmem_base + (uint32_t)((acc * MT + j) * BN), quad, lane, ms * MT + j, nt, wo);
+        if (mask & (1 << j)) epilogue_tile<EPI>(p, tmem_base + (uint32_t)((acc * MT + j) * BN), quad, lane, ms * MT + j, nt, wo);
       tc_fence_before();
       mbar_arrive(tempty_bar(acc));
       if (++acc == NACC) { acc = 0; acc_phase ^= 1u; }
@@ -644,7 +667,7 @@ cudaError_t launch_tc_gemm(const TcGemm& g, cudaStream_t s) {
   a.ids = g.ids; a.lse = g.lse; a.g = g.g; a.partials = g.partials; a.tgt = g.tgt;
   a.dS = g.dS; a.ds_ld = g.ds_ld;
   a.dHidden = g.dHidden; a.dh_ld = g.dh_ld; a.dW = g.dW; a.dw_ld = g.dw_ld; a.status = g.status;
-  a.psum = g.psum; a.row_scale = g.row_scale;
+  a.psum = g.psum; a.row_scale = g.row_scale; a.blk_active = g.blk_active;
   const int NT = cdiv(g.N, BN);
   const int mt = (g.epi == TC_EPI_DW || g.epi == TC_EPI_DH) ? 2 : 1;
   const long max_tiles = (long)cdiv(g.epi == TC_EPI_DW ? g.m_blocks : g.blk_cap, mt) * NT;

@@ -60,6 +60,8 @@ CONFIGS = {
     2: Workload("cfg2_8b_fwdbwd", P=8, G=8, T=2048, H=4096, V=151936),
     3: Workload("cfg3_long_reasoning", P=4, G=8, T=8192, H=4096, V=151936,
                 len_lo=0.125, bnd_lo=0.5, bnd_hi=0.9),
+    # one representative point of the config-4 sweep (the full grid is sweep_workloads())
+    4: Workload("cfg4_V151936_H4096_G8", P=8, G=8, T=1024, H=4096, V=151936, degenerate_frac=0.25),
     # not one of the five: a few-GB case of the same kernels for profiler captures
     5: Workload("profile_small", P=1, G=8, T=2048, H=4096, V=32768),
 }
