@@ -93,7 +93,8 @@ size_t trl_workspace_bytes_min(int which_call, int B, int T, int H, int V, trl_d
  *   z[n,v] = sum_k hidden[n,k] W[v,k];  lse[n] = log sum_v exp z[n,v];  logp[n] = z[n,ids[n]] - lse[n]
  *
  * The [N,V] logits are never written to memory (bf16 path: vocabulary tiles are reduced
- * to a running (max, sum-exp) pair in the GEMM epilogue).
+ * to a running (max, sum-exp) pair in the GEMM epilogue).  The workspace holds a packed copy
+ * of the valid rows of `hidden` and the per-tile partials.
  *
  * in : hidden [B*T,H] dt; W [V,H] dt; ids [B*T] int32; len [B] int32
  * out: logp [B*T] f32; lse [B*T] f32 (save lse for trl_pg_loss_bwd)

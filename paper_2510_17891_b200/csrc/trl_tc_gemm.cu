@@ -1,7 +1,7 @@
 // tcgen05 / TMEM bf16 GEMM family for sm_100a.
 //
 // One persistent, warp-specialised kernel computes C[m,n] = sum_k A[m,k] B[n,k] (bf16
-// operands, fp32 accumulation in tensor memory) on 128x256 tiles.  Each operand is read in
+// operands, fp32 accumulation in tensor memory) on 128x256 accumulator tiles.  Each operand is read in
 // the layout it already has in memory: K-contiguous ("K-major": hidden and W in the forward,
 // dS / E in dHidden = dS W) or M/N-contiguous ("MN-major": W in dHidden = dS W, dS / E and the
 // gathered hidden rows in dW = dS^T hidden), so no operand is ever transposed in memory.
@@ -11,9 +11,10 @@
 //   DS  : dS = g (onehot - exp(z - lse)) as bf16
 //   DH  : dHidden rows (bf16), scattered to the caller's row positions
 //   DW  : dW += tile (fp32, TMA reduce-add from shared memory)
-//   E   : E = exp(z - c) for a per-row shift c (a stale log-partition), as bf16, plus the row sums of E and the sampled token's logit.  The softmax
-//         is p = E exp(c - lse), a per-row factor the gradient GEMMs fold into their other
-//         operand / their epilogue, so the forward GEMM is not repeated in the backward.
+//   E   : E = exp(z - c) for a per-row shift c (a stale log-partition), as bf16, plus the row
+//         sums of E and the sampled token's logit.  The softmax is p = E exp(c - lse), a
+//         per-row factor the gradient GEMMs fold into their other operand / their epilogue,
+//         so the forward GEMM is not repeated in the backward.
 //
 // Roles: warp 0 = TMA producer (one elected lane), warp 1 = MMA issuer (one elected lane)
 // and TMEM owner, warps 2..5 = epilogue (one TMEM lane quadrant each).  Shared-memory
