@@ -140,6 +140,51 @@ def run_reference(args, rank, world):
     print(json.dumps(line))
 
 
+def run_reductions(trl, torch, dev, peaks, args):
+    """HBM roofline of the memory-bound calls at a size where launch latency no longer hides it:
+    512 rollouts x 131,072 tokens = 2^26 tokens (the benchmark configs move < 5 MB through them)."""
+    P, G, T = 64, 8, 131072
+    B, N = P * G, P * G * T
+    g = torch.Generator(device=dev).manual_seed(1)
+    lens = torch.randint(T // 4, T + 1, (B,), generator=g, device=dev, dtype=torch.int32)
+    bnd = (lens.float() * (0.2 + 0.6 * torch.rand(B, generator=g, device=dev))).to(torch.int32)
+    r_plan = (torch.rand(B, generator=g, device=dev) < 0.3).float()
+    r_code = (torch.rand(B, generator=g, device=dev) < 0.6).float()
+    old = -torch.rand(N, generator=g, device=dev) * 5
+    logp = old + 0.05 * torch.randn(N, generator=g, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    hrd = trl.trl_hrd_advantages(r_plan, r_code, lens, bnd, P, G, T, status=status)
+    loss, gg, stats = trl.trl_pg_loss_fwd(logp, old, hrd["adv"], hrd["seg"], lens, P, G, T, status=status)
+    ws = torch.empty(trl.trl_workspace_bytes(trl.TRL_CALL_PG_LOSS_FWD, B, T, 1, 1, trl.TRL_F32), dtype=torch.uint8, device=dev)
+    n_valid = int(lens.sum())
+
+    def timed(fn, n=20):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(n):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / n
+
+    t_adv = timed(lambda: trl.trl_hrd_advantages(r_plan, r_code, lens, bnd, P, G, T, 0, hrd, status))
+    t_loss = timed(lambda: trl.trl_pg_loss_fwd(logp, old, hrd["adv"], hrd["seg"], lens, P, G, T, 0.2, 0.2, 0.1,
+                                               loss, gg, stats, ws, status))
+    trl.check_status(status)
+    # algorithmic bytes: advantages write seg (1 B) + adv (4 B) per padded token; the loss reads
+    # logp, old_logp, adv (12 B) + seg (1 B) per valid token and writes g (4 B) per padded token
+    b_adv = 5.0 * N
+    b_loss = 13.0 * n_valid + 4.0 * N
+    line = dict(metric="reduction_kernels_hbm", tokens=N, valid_tokens=n_valid,
+                hrd_advantages=dict(ms=t_adv, bytes=b_adv, gbs=b_adv / t_adv / 1e6, frac=b_adv / t_adv / 1e6 / peaks["hbm_gbs"]),
+                pg_loss_fwd=dict(ms=t_loss, bytes=b_loss, gbs=b_loss / t_loss / 1e6, frac=b_loss / t_loss / 1e6 / peaks["hbm_gbs"]),
+                peak_gbs=peaks["hbm_gbs"], peak_source=peaks["source"] + " copy bandwidth")
+    print(json.dumps(line))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -148,6 +193,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", type=int, default=WORKLOAD_ID, help="config number (default: the metric's)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--reductions", action="store_true",
+                    help="time the two memory-bound calls (HRD advantages, surrogate loss) alone at 2^26 tokens")
     ap.add_argument("--path", default="fused", choices=["fused", "four_call"],
                     help="fused: old-policy scoring, advantages, trl_pg_step_fused; four_call: the separate calls")
     args = ap.parse_args()
@@ -172,8 +219,11 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
 
-    w = synth.CONFIGS[args.workload]
     peaks = load_peaks()
+    if args.reductions:
+        run_reductions(trl, torch, dev, peaks, args)
+        return
+    w = synth.CONFIGS[args.workload]
     batch = synth.make_batch(w, device=dev, seed_offset=dp.rank_seed_offset(rank))
     batch["hidden_old"] = batch["hidden"].clone()        # the old policy's own activation buffer
     B, T, H, V, P, G = w.B, w.T, w.H, w.V, w.P, w.G

@@ -204,7 +204,7 @@ int trl_pg_step_fused(const void* hidden, const void* W, const int32_t* ids, con
  * counterpart to this call; it exists for such callers only.)
  *
  * The partial sums live in a fixed 1 MiB array inside the library image (every GPU that
- * loads the library holds it until the process exits).  Limit: P*G*ceil(T/4096) <= 65536,
+ * loads the library holds it until the process exits).  Limit: P*G*ceil(T/16384) <= 65536,
  * otherwise TRL_ERR_WORKSPACE_TOO_SMALL is returned and nothing is launched.  The call
  * performs no cudaMalloc / cudaFree and calls no allocating routine; inputs and outputs are
  * still the caller's device buffers.

@@ -181,7 +181,7 @@ def trl_pg_loss_fwd_static(logp, old_logp, adv, seg, lens, P, G, T, loss, g, sta
                            alpha=0.1, status=None, stream=None, clip_form=0, agg_mode=0):
     """trl_pg_loss_fwd for callers that cannot allocate: the scratch is a fixed array inside the
     library, and this wrapper allocates nothing either, so `loss` [1], `g` [P*G*T] and `stats`
-    [4] (or None) must be passed in.  Limit P*G*ceil(T/4096) <= 65536.  Calls that may overlap
+    [4] (or None) must be passed in.  Limit P*G*ceil(T/16384) <= 65536.  Calls that may overlap
     on the GPU must not share a device.  Returns (loss, g, stats)."""
     _dev(logp, old_logp, adv, seg, lens, loss, g, stats, status)
     rc = load_library().trl_pg_loss_fwd_static(_ptr(logp), _ptr(old_logp), _ptr(adv), _ptr(seg), _ptr(lens), P, G, T,

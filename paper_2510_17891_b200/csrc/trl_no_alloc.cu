@@ -47,7 +47,7 @@ extern "C" int trl_pg_loss_fwd_static(const float* logp, const float* old_logp, 
   if (P <= 0 || G <= 0 || T <= 0 || (long)P * G > 65535 || (long)P * G * T >= (1L << 31)) return TRL_ERR_SHAPE;
   if (!(cfg.eps_lo >= 0.f) || !(cfg.eps_hi >= 0.f) || !(cfg.alpha >= 0.f) || (cfg.clip_form & ~1) || (cfg.agg_mode & ~1))
     return TRL_ERR_INVALID_ARG;
-  // size limit of the built-in scratch: P*G*ceil(T/4096) slots
+  // size limit of the built-in scratch: P*G*ceil(T/16384) slots
   if ((long)P * G * trl::pg_loss_tiles(T) > kStaticLossSlots) return TRL_ERR_WORKSPACE_TOO_SMALL;
   int major = 0, dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess ||

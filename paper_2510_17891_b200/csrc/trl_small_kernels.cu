@@ -144,23 +144,29 @@ __global__ void __launch_bounds__(256) hrd_adv_kernel(
   const int L = s_lb[0], Bd = s_lb[1];
   const int t_begin = blockIdx.x * kAdvTile, t_end = min(T, t_begin + kAdvTile);
   const size_t base = (size_t)b * T;
-  // 16 tokens per thread-iteration when the row start is 16-aligned, else scalar
+  // A warp covers 512 consecutive tokens per iteration when rows are 16-aligned.  Every store
+  // instruction of the warp writes 512 contiguous bytes: lane i writes the 16 segment bytes of
+  // tokens [16i, 16i+16), and for q = 0..3 the four advantages of tokens [128q + 4i, 128q + 4i + 4).
   if ((T & 15) == 0) {
-    for (int t = t_begin + tid * 16; t < t_end; t += 256 * 16) {
+    const int lane = tid & 31, wid = tid >> 5;
+    for (int t0 = t_begin + wid * 512; t0 < t_end; t0 += 8 * 512) {
       uint32_t w[4];
-      float a[16];
 #pragma unroll
       for (int q = 0; q < 16; ++q) {
-        const int tt = t + q;
+        const int tt = t0 + lane * 16 + q;
         const int sg = tt < Bd ? 1 : (tt < L ? 2 : 0);
-        a[q] = sg == 1 ? ap : (sg == 2 ? ac : 0.f);
         if ((q & 3) == 0) w[q >> 2] = 0;
         w[q >> 2] |= (uint32_t)sg << (8 * (q & 3));
       }
-      *reinterpret_cast<uint4*>(seg + base + t) = make_uint4(w[0], w[1], w[2], w[3]);
+      if (t0 + lane * 16 < t_end) *reinterpret_cast<uint4*>(seg + base + t0 + lane * 16) = make_uint4(w[0], w[1], w[2], w[3]);
 #pragma unroll
-      for (int q = 0; q < 4; ++q)
-        *reinterpret_cast<float4*>(adv + base + t + 4 * q) = make_float4(a[4 * q], a[4 * q + 1], a[4 * q + 2], a[4 * q + 3]);
+      for (int q = 0; q < 4; ++q) {
+        const int tt = t0 + 128 * q + 4 * lane;
+        float a[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) a[k] = (tt + k) < Bd ? ap : ((tt + k) < L ? ac : 0.f);
+        if (tt < t_end) *reinterpret_cast<float4*>(adv + base + tt) = make_float4(a[0], a[1], a[2], a[3]);
+      }
     }
   } else {
     for (int t = t_begin + tid; t < t_end; t += 256) {
@@ -186,7 +192,7 @@ void launch_hrd_advantages(const float* r_plan, const float* r_code, const int32
 // rollout in a fixed order and writes 4 partial sums; also writes g.  Stage 2: one CTA
 // combines the partials in index order in fp64 -> bit-reproducible loss.
 // ------------------------------------------------------------------------------------
-constexpr int kLossTile = 4096;
+constexpr int kLossTile = 16384;
 int pg_loss_tiles(int T) { return cdiv(T, kLossTile); }
 
 // One token of the surrogate: returns w*u and writes s and g (before the 1/normaliser factor
@@ -240,18 +246,45 @@ __global__ void __launch_bounds__(256) pg_loss_stage1_kernel(
   }
   const float lo = 1.0f - cfg.eps_lo, hi = 1.0f + cfg.eps_hi;
   float acc = 0.f, n_hi = 0.f, n_lo = 0.f, sum_s = 0.f;
-  for (int t = t_begin + tid; t < t_end; t += 256) {
-    float gn = 0.f;
-    if (t < L) {
-      const size_t n = base + t;
-      const TokenTerm tt = surrogate_token(logp[n], old_logp[n], adv[n], seg[n], cfg, inv);
-      acc += tt.wu;
-      gn = tt.g;
-      n_hi += tt.s > hi ? 1.f : 0.f;
-      n_lo += tt.s < lo ? 1.f : 0.f;
-      sum_s += tt.s;
+  if ((T & 3) == 0) {          // 4 tokens per thread: 16-byte loads and stores
+    for (int t = t_begin + tid * 4; t < t_end; t += 256 * 4) {
+      float gq[4] = {0.f, 0.f, 0.f, 0.f};
+      if (t < L) {
+        const size_t n = base + t;
+        const float4 lp = *reinterpret_cast<const float4*>(logp + n);
+        const float4 ol = *reinterpret_cast<const float4*>(old_logp + n);
+        const float4 ad = *reinterpret_cast<const float4*>(adv + n);
+        const uchar4 sg = *reinterpret_cast<const uchar4*>(seg + n);
+        const float lpa[4] = {lp.x, lp.y, lp.z, lp.w}, ola[4] = {ol.x, ol.y, ol.z, ol.w}, ada[4] = {ad.x, ad.y, ad.z, ad.w};
+        const int sga[4] = {sg.x, sg.y, sg.z, sg.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          if (t + k < L) {
+            const TokenTerm tt = surrogate_token(lpa[k], ola[k], ada[k], sga[k], cfg, inv);
+            acc += tt.wu;
+            gq[k] = tt.g;
+            n_hi += tt.s > hi ? 1.f : 0.f;
+            n_lo += tt.s < lo ? 1.f : 0.f;
+            sum_s += tt.s;
+          }
+        }
+      }
+      *reinterpret_cast<float4*>(g + base + t) = make_float4(gq[0], gq[1], gq[2], gq[3]);
     }
-    g[base + t] = gn;
+  } else {
+    for (int t = t_begin + tid; t < t_end; t += 256) {
+      float gn = 0.f;
+      if (t < L) {
+        const size_t n = base + t;
+        const TokenTerm tt = surrogate_token(logp[n], old_logp[n], adv[n], seg[n], cfg, inv);
+        acc += tt.wu;
+        gn = tt.g;
+        n_hi += tt.s > hi ? 1.f : 0.f;
+        n_lo += tt.s < lo ? 1.f : 0.f;
+        sum_s += tt.s;
+      }
+      g[base + t] = gn;
+    }
   }
   __shared__ float red[4][8];
   float v[4] = {acc, n_hi, n_lo, sum_s};
@@ -268,35 +301,42 @@ __global__ void __launch_bounds__(256) pg_loss_stage1_kernel(
   }
 }
 
+// One CTA.  Thread b adds its rollouts' tile partials in tile order (independent loads),
+// divides by the length, and the block combines the per-thread fp64 sums in a fixed tree.
 __global__ void __launch_bounds__(256) pg_loss_stage2_kernel(const float* __restrict__ partials,
                                                              const int32_t* __restrict__ len, int P, int G, int T,
                                                              int tiles, int agg_mode, float* __restrict__ loss,
                                                              float* __restrict__ stats) {
-  __shared__ double red[4][256];
-  const int tid = threadIdx.x, B = P * G;
-  double J = 0, nh = 0, nl = 0, ss = 0;
+  __shared__ double red[5][8];
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5, B = P * G;
+  double v[5] = {0, 0, 0, 0, 0};          // J, n_hi, n_lo, sum_s, tokens
   for (int b = tid; b < B; b += 256) {
     const int L = max(0, min(len[b], T));
+    const float4* p4 = reinterpret_cast<const float4*>(partials) + (size_t)b * tiles;
     double a = 0;
+#pragma unroll 8
     for (int k = 0; k < tiles; ++k) {
-      const float* p = partials + ((size_t)b * tiles + k) * 4;
-      a += p[0]; nh += p[1]; nl += p[2]; ss += p[3];
+      const float4 p = p4[k];
+      a += p.x; v[1] += p.y; v[2] += p.z; v[3] += p.w;
     }
-    if (L > 0) J += agg_mode == 1 ? a : a / L;
+    if (L > 0) v[0] += agg_mode == 1 ? a : a / L;
+    v[4] += L;
   }
-  red[0][tid] = J; red[1][tid] = nh; red[2][tid] = nl; red[3][tid] = ss;
+#pragma unroll
+  for (int q = 0; q < 5; ++q) {
+    for (int o = 16; o > 0; o >>= 1) v[q] += __shfl_xor_sync(0xffffffffu, v[q], o);
+    if (lane == 0) red[q][wid] = v[q];
+  }
   __syncthreads();
   if (tid == 0) {
-    double t[4] = {0, 0, 0, 0};
-    for (int q = 0; q < 4; ++q)
-      for (int k = 0; k < 256; ++k) t[q] += red[q][k];
-    long long ntok = 0;
-    for (int b = 0; b < B; ++b) ntok += max(0, min(len[b], T));
-    loss[0] = agg_mode == 1 ? (float)(ntok > 0 ? -t[0] / (double)ntok : 0.0) : (float)(-t[0] / ((double)P * (double)G));
+    double t[5] = {0, 0, 0, 0, 0};
+    for (int q = 0; q < 5; ++q)
+      for (int k = 0; k < 8; ++k) t[q] += red[q][k];
+    loss[0] = agg_mode == 1 ? (float)(t[4] > 0 ? -t[0] / t[4] : 0.0) : (float)(-t[0] / ((double)P * (double)G));
     if (stats) {
-      const double d = ntok > 0 ? (double)ntok : 1.0;
+      const double d = t[4] > 0 ? t[4] : 1.0;
       stats[0] = (float)(t[1] / d); stats[1] = (float)(t[2] / d); stats[2] = (float)(t[3] / d);
-      stats[3] = (float)ntok;
+      stats[3] = (float)t[4];
     }
   }
 }

@@ -45,7 +45,7 @@ def test_static_scratch_variant_matches_workspace_variant_twice_in_a_row():
 
 def test_static_scratch_variant_rejects_oversize():
     import paper_2510_17891_b200 as trl
-    P, G, T = 1, 60000, 8192          # 60000 * 2 tiles > 65536 slots
+    P, G, T = 1, 60000, 32768         # 60000 * 2 tiles > 65536 slots
     dummy = torch.zeros(8, device="cuda")
     with pytest.raises(trl.TrlError, match="workspace too small"):
         trl.trl_pg_loss_fwd_static(dummy, dummy, dummy, dummy.to(torch.uint8), dummy.to(torch.int32), P, G, T,
