@@ -47,7 +47,10 @@ size_t fwd_bytes_bf16(int B, int T, int H, int V) { return row_pack_bytes(B, T) 
 size_t fwd_bytes_f32(int B, int T, int H, int V, int R) {
   return row_pack_bytes(B, T) + align_up((size_t)R * H * 4, 256) + align_up((size_t)R * V * 4, 256);
 }
-size_t bwd_fixed_bf16(int B, int T, int H, int V) { (void)V; return row_pack_bytes(B, T) + xp_bytes(B, T, H); }
+size_t bwd_fixed_bf16(int B, int T, int H, int V) {     // row packing, packed hidden, row-block activity flags
+  (void)V;
+  return row_pack_bytes(B, T) + xp_bytes(B, T, H) + align_up((size_t)cdiv(B * T, kRowBlock) * 4, 256);
+}
 size_t bwd_per_rows_bf16(int H, int V, int R) { (void)H; return align_up((size_t)R * V * 2, 256); }   // dS chunk
 size_t bwd_bytes_f32(int B, int T, int H, int V, int R) {
   return row_pack_bytes(B, T) + 2 * align_up((size_t)R * H * 4, 256) + align_up((size_t)R * V * 4, 256);
@@ -242,13 +245,15 @@ int trl_pg_loss_bwd(const void* hidden, const void* W, const int32_t* ids, const
                            [&](int r) { return bwd_per_rows_bf16(H, V, r); });
     if (R < kRowBlock) return TRL_ERR_WORKSPACE_TOO_SMALL;
     __nv_bfloat16* Xp = cv.take<__nv_bfloat16>((size_t)cap_rows * H);
+    int* blk_active = cv.take<int>(rb.cap);
     __nv_bfloat16* dS = cv.take<__nv_bfloat16>((size_t)R * V);
     launch_pack_rows_bf16((const __nv_bfloat16*)hidden, Xp, H, cap_rows, rb, 0, 0, nullptr, s);
+    launch_flag_active_blocks(g, rb, blk_active, s);     // row blocks with g == 0 everywhere are skipped below
     const int CB = R / kRowBlock;
     for (int blk_off = 0; blk_off < rb.cap; blk_off += CB) {
       TcGemm a;
       memset(&a, 0, sizeof(a));
-      a.rb = rb; a.blk_off = blk_off; a.blk_cap = CB; a.status = status_dev;
+      a.rb = rb; a.blk_off = blk_off; a.blk_cap = CB; a.status = status_dev; a.blk_active = blk_active + blk_off;
       // dS chunk = g (onehot - softmax), from a recomputed logits tile
       TcGemm ds = a;
       ds.epi = TC_EPI_DS; ds.raster_band = kRasterBandFwdE;

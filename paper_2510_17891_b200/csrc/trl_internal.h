@@ -62,6 +62,8 @@ struct FusedMergeArgs {
   int32_t* status;
 };
 void launch_fused_merge(const FusedMergeArgs& a, cudaStream_t s);
+// blk_active[i] = 1 if any of the 128 packed rows of row block i has g != 0 (i < nblk)
+void launch_flag_active_blocks(const float* g, RowPack rb, int* blk_active, cudaStream_t s);
 // fp32 path helpers
 void launch_pack_rows_f32(const float* hidden, float* Xp, int H, int R, RowPack rb, int blk_off, cudaStream_t s);
 void launch_row_lse_f32(const float* S, int V, int R, RowPack rb, int blk_off, const int32_t* ids,
@@ -108,7 +110,7 @@ struct TcGemm {
   float* dW; long dw_ld; int V;                        // DW
   float* psum;                                         // E: row sums per vocabulary tile [n_tiles, rows_cap]
   const float* row_scale;                              // DH: optional per-scratch-row factor
-  const int* blk_active;                               // DH, DW: optional per-row-block activity flags of the chunk
+  const int* blk_active;                               // DS, DH, DW: optional per-row-block activity flags of the chunk
   int32_t* status;
 };
 // returns cudaSuccess or the error of tensor-map creation / launch

@@ -479,6 +479,20 @@ __global__ void __launch_bounds__(128) fused_merge_kernel(FusedMergeArgs a) {
   if (threadIdx.x == 0) a.blk_active[blockIdx.x] = any;
 }
 
+__global__ void __launch_bounds__(128) flag_active_blocks_kernel(const float* __restrict__ g, RowPack rb,
+                                                                 int* __restrict__ blk_active) {
+  if ((int)blockIdx.x >= rb.nblk[0]) return;
+  const int q = blockIdx.x * kRowBlock + threadIdx.x;
+  const bool on = q < rb.n_rows[0] && g[rb.rowmap[q]] != 0.f;
+  const int any = __syncthreads_or(on);
+  if (threadIdx.x == 0) blk_active[blockIdx.x] = any;
+}
+
+void launch_flag_active_blocks(const float* g, RowPack rb, int* blk_active, cudaStream_t s) {
+  flag_active_blocks_kernel<<<rb.cap, 128, 0, s>>>(g, rb, blk_active);
+  note_launch();
+}
+
 void launch_fused_merge(const FusedMergeArgs& a, cudaStream_t s) {
   fused_merge_kernel<<<cdiv(a.R, 128), 128, 0, s>>>(a);
   note_launch();

@@ -425,12 +425,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   }
   if (total == 0 || (int)blockIdx.x >= total) return;
   // Which M sub-blocks of a CTA tile take part (identical decision in every role): present, and for
-  // dHidden not marked inactive.  Which k-blocks take part: for dW, those of active row blocks.
+  // dS / dHidden not marked inactive.  Which k-blocks take part: for dW, those of active row blocks.
   auto tile_mask = [&](int ms) {
     const int nm = min(MT, MB - ms * MT);
     int m = 0;
     for (int j = 0; j < nm; ++j)
-      if (!(EPI == TC_EPI_DH && p.blk_active) || p.blk_active[ms * MT + j] != 0) m |= 1 << j;
+      if (!((EPI == TC_EPI_DH || EPI == TC_EPI_DS) && p.blk_active) || p.blk_active[ms * MT + j] != 0) m |= 1 << j;
     return m;
   };
   auto kb_on = [&](int kb) { return !(EPI == TC_EPI_DW && p.blk_active) || p.blk_active[kb >> 1] != 0; };

@@ -251,6 +251,17 @@ def test_fused_step_minimum_workspace_chunks(trl):
     assert rel_fro(f64(out["dW"]), f64(ref["dW"])) < 1e-5
 
 
+@pytest.mark.parametrize("fused", [False, True])
+def test_many_rollouts_and_odd_length(trl, fused):
+    """More rollouts than the threads of the row-packing scan (1024), and a T that is not a multiple
+    of 4 (scalar paths of the advantage / loss kernels, rollouts that do not start 16-byte aligned)."""
+    w = synth.scaled(synth.CONFIGS[2], name="many_rollouts", P=150, G=8, T=12, H=64, V=256, len_lo=0.0)
+    run_and_compare(trl, w, fused=fused)
+    w = synth.scaled(synth.CONFIGS[2], name="odd_T", P=2, G=3, T=75, H=128, V=520, len_lo=0.3)
+    run_and_compare(trl, w, fused=fused)
+    run_and_compare(trl, synth.scaled(w, name="odd_T_f32", dtype="f32"), fused=fused)
+
+
 def test_minimum_workspace_gives_same_backward(trl):
     # chunked backward (one 128-row block per chunk) equals the one-chunk result
     w = synth.scaled(synth.CONFIGS[2], name="chunks", P=1, G=3, T=200, H=128, V=512)
