@@ -381,9 +381,9 @@ def main():
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        v_cpu, tok, sec, threads = oracle_sample_throughput(w, 8, 48)
+        v_cpu, tok, sec, threads = oracle_sample_throughput(w, 12, 64)
         cpu_baseline = dict(value=v_cpu, unit=UNIT, cores=threads, kind="oracle",
-                            sample=f"8 rollouts x T=48 ({tok} valid tokens, {sec:.1f} s), full H={H} V={V}, whole path in numpy fp64")
+                            sample=f"12 rollouts x T=64 ({tok} valid tokens, {sec:.1f} s), full H={H} V={V}, whole path in numpy fp64")
 
     if rank == 0:
         line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=max(args.warmup, 3),

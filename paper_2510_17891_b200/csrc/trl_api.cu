@@ -24,7 +24,7 @@ int check_device() {
 }
 
 bool shapes_ok(int B, int T, int H, int V) {
-  return B > 0 && T > 0 && H > 0 && V > 0 && (long)B * T < (1L << 31) && (long)V * H < (1L << 40);
+  return B > 0 && T > 0 && H > 0 && V > 0 && (long)B * T < (1L << 31) - 256 && (long)V * H < (1L << 40);
 }
 
 struct Carver {
