@@ -195,6 +195,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--reductions", action="store_true",
                     help="time the two memory-bound calls (HRD advantages, surrogate loss) alone at 2^26 tokens")
+    ap.add_argument("--dp-allreduce", action="store_true",
+                    help="N > 1 only: also all-reduce dW and the loss across ranks every step (data-parallel training)")
     ap.add_argument("--path", default="fused", choices=["fused", "four_call"],
                     help="fused: old-policy scoring, advantages, trl_pg_step_fused; four_call: the separate calls")
     args = ap.parse_args()
@@ -279,7 +281,12 @@ def main():
                             bufs["dHidden"], bufs["dW"], bufs["ws_bwd"], status, stream)
         mark()
 
-    step = step_fused if args.path == "fused" else step_four
+    step_local = step_fused if args.path == "fused" else step_four
+
+    def step(ev=None, batch=batch):
+        step_local(ev, batch)
+        if args.dp_allreduce and dist is not None:
+            dp.allreduce_step_outputs(bufs["dW"], bufs["loss"], P)
 
     def _rec():
         e = torch.cuda.Event(enable_timing=True)
@@ -391,7 +398,8 @@ def main():
                     dtype=w.dtype, data="synthetic",
                     config=dict(workload=w.name, P=P, G=G, T=T, H=H, V=V, valid_tokens_per_rank=n_valid,
                                 padded_rows_per_rank=B * T, l2="inputs larger than L2 (W alone is 1.2 GB); no flush",
-                                parallelism=f"replicas x{world} (independent batches)"),
+                                parallelism=(f"data-parallel x{world}, dW + loss all-reduced every step" if args.dp_allreduce and world > 1
+                                             else f"replicas x{world} (independent batches)")),
                     pct_of_bf16_peak_6NHV=dict(sustained=100 * step_alg / peaks["bf16_sustained"],
                                                burst=100 * step_alg / peaks["bf16_burst"], nominal=100 * step_alg / 2250.0,
                                                note="6*H*V FLOP per scored token over the whole step (which also scores the old policy)"),

@@ -1,8 +1,13 @@
 """Data-parallel plumbing for N > 1 ranks (one process per GPU).
 
 The path shards by prompt group: every rank scores its own rollout groups with its own copy
-of the LM head, so the data path has no exchange step; only the benchmark's bookkeeping
-(time = max over ranks, tokens = sum over ranks) crosses ranks."""
+of the LM head, so scoring, advantages, loss and backward have no exchange step.  What a
+data-parallel trainer exchanges afterwards is the LM-head gradient (and the scalar loss):
+`allreduce_step_outputs` does that with the process group's all-reduce (NCCL over NVLink on
+GPUs, gloo on CPU), in buckets so the first buckets can be reduced while later ones are
+still being enqueued.  The benchmark keeps it off by default (ranks are independent
+replicas there); its bookkeeping (time = max over ranks, tokens = sum) is in
+`aggregate_throughput`."""
 import torch
 import torch.distributed as dist
 
@@ -23,3 +28,27 @@ def aggregate_throughput(elapsed_ms: float, tokens_per_step: int, steps: int, de
         dist.all_reduce(n, op=dist.ReduceOp.SUM)
         elapsed_ms, tokens_per_step = float(t.item()), int(n.item())
     return tokens_per_step * steps / (elapsed_ms * 1e-3), elapsed_ms, tokens_per_step
+
+
+def allreduce_step_outputs(dW: torch.Tensor, loss: torch.Tensor, n_prompts_local: int, bucket_bytes: int = 256 << 20):
+    """Combine the per-rank results of one step into the global-batch gradient and loss, in place.
+
+    Each rank computed its loss as a mean over its own P_r prompts, so the global mean over
+    sum_r P_r prompts is sum_r (P_r / P_total) * loss_r, and the same weights apply to dW.
+    dW is reduced bucket by bucket with asynchronous all-reduces; the call returns when all of
+    them have completed on the current stream.  Without a process group it is the identity.
+    Returns the global number of prompts."""
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return n_prompts_local
+    tot = torch.tensor([float(n_prompts_local)], dtype=torch.float64, device=dW.device)
+    dist.all_reduce(tot, op=dist.ReduceOp.SUM)
+    weight = n_prompts_local / float(tot.item())
+    flat = dW.view(-1)
+    flat.mul_(weight)
+    loss.mul_(weight)
+    step = max(1, bucket_bytes // flat.element_size())
+    works = [dist.all_reduce(flat[i:i + step], op=dist.ReduceOp.SUM, async_op=True) for i in range(0, flat.numel(), step)]
+    works.append(dist.all_reduce(loss, op=dist.ReduceOp.SUM, async_op=True))
+    for wk in works:
+        wk.wait()
+    return int(round(tot.item()))
