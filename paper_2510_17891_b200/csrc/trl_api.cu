@@ -13,14 +13,16 @@ constexpr int kRasterBandFwd = 32;
 constexpr int kRasterBandFwdE = 24;   // forward tiles that also store E / dS
 constexpr int kRasterBandBwd = 4;
 
-int check_device() {
-  static int cached = -1;
-  if (cached >= 0) return cached;
+int check_device() {      // the current device must be compute capability 10.x (cached per device)
+  static int cached[64];
+  static bool known[64] = {};
   int dev = 0, major = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess) return TRL_ERR_CUDA;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return TRL_ERR_CUDA;
+  if (known[dev]) return cached[dev];
   if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return TRL_ERR_CUDA;
-  cached = (major == 10) ? TRL_OK : TRL_ERR_ARCH;
-  return cached;
+  cached[dev] = (major == 10) ? TRL_OK : TRL_ERR_ARCH;
+  known[dev] = true;
+  return cached[dev];
 }
 
 bool shapes_ok(int B, int T, int H, int V) {
