@@ -28,7 +28,7 @@ UNIT = "tokens/s"
 WORKLOAD_ID = 2          # 8B-scale fwd+bwd: 8 prompts x 8 rollouts, T=2048, H=4096, V=151,936
 # DRAM bytes (read + write) of one tc_gemm_kernel<LSE> launch at WORKLOAD_ID, from the ncu capture of
 # the same kernel on the profile_small workload (0.897 GB: packed hidden once + W once per raster
-# band of 32 row blocks), scaled by (bands x bytes of W): see profiles/tc_gemm_profile_small_ncu_full.md
+# band of 32 row blocks), scaled by (bands x bytes of W); the capture's summary is committed under profiles/
 LSE_TRAFFIC_BYTES = 2.85e10
 
 
