@@ -114,21 +114,36 @@ def oracle_sample_throughput(w, rollouts, T_sample, seed_offset=0):
 
 
 def run_reference(args, rank, world):
-    """Reference arm = the oracle on the host cores (rank 0 only)."""
+    """Reference arm = the oracle on the host cores (rank 0 only).  One batch of short rollouts
+    with the full H and V is drawn once; every step runs the whole path on two of them."""
     if rank != 0:
         return
+    import torch
+    from threadpoolctl import threadpool_info
+    from oracle import trl_oracle as orc
     from paper_2510_17891_b200 import synth
     w = synth.CONFIGS[WORKLOAD_ID]
-    rollouts, T_sample = 2, 16
-    for i in range(args.warmup):
-        oracle_sample_throughput(w, 1, 4, seed_offset=100 + i)
-    tok = sec = 0
-    threads = 1
-    for i in range(args.steps):
-        _, t, s, threads = oracle_sample_throughput(w, rollouts, T_sample, seed_offset=i)
-        tok += t; sec += s
+    per_step, T_sample = 2, 16
+    n_steps = args.steps + args.warmup
+    ws = synth.scaled(w, name=w.name + "_cpu_reference", P=n_steps, G=per_step, T=T_sample)
+    b = synth.make_batch(ws, device="cpu")
+    f64 = lambda t: t.to(torch.float64).numpy()
+    W, W_old, hidden = f64(b["W"]), f64(b["W_old"]), f64(b["hidden"])
+    ids, lens, bnd = b["ids"].numpy(), b["lens"].numpy(), b["bnd"].numpy()
+    rp, rc = f64(b["r_plan"]), f64(b["r_code"])
+    tok = 0
+    sec = 0.0
+    for i in range(n_steps):
+        r = slice(i * per_step, (i + 1) * per_step)
+        rows = slice(i * per_step * T_sample, (i + 1) * per_step * T_sample)
+        t0 = time.perf_counter()
+        orc.full_step(hidden[rows], W, hidden[rows], W_old, ids[rows], lens[r], bnd[r], rp[r], rc[r], 1, per_step, T_sample)
+        dt = time.perf_counter() - t0
+        if i >= args.warmup:
+            tok += int(lens[r].sum()); sec += dt
+    threads = max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
     value = tok / sec
-    sample = (f"{rollouts} rollouts x T={T_sample} per step (valid tokens only), full H={w.H} V={w.V}, "
+    sample = (f"{per_step} rollouts x T={T_sample} per step (valid tokens only), full H={w.H} V={w.V}, "
               f"policy + old-policy scoring, advantages, loss, backward in numpy fp64")
     line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps, warmup=args.warmup,
                 ms_per_step=1e3 * sec / max(args.steps, 1), higher_is_better=True, scaling="weak", vs_baseline=None,
