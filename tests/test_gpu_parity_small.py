@@ -262,6 +262,17 @@ def test_many_rollouts_and_odd_length(trl, fused):
     run_and_compare(trl, synth.scaled(w, name="odd_T_f32", dtype="f32"), fused=fused)
 
 
+@pytest.mark.parametrize("shape", [(1, 1, 1, 8, 8), (1, 2, 3, 8, 1000), (2, 2, 5, 1024, 8), (1, 3, 130, 16, 24),
+                                   (1, 1, 128, 64, 256), (1, 1, 129, 64, 264)])
+def test_smallest_legal_shapes(trl, shape):
+    """Tensors smaller than one TMA box / one tile in every dimension (H = V = 8, T = 1), and shapes
+    one past a tile edge."""
+    P, G, T, H, V = shape
+    w = synth.scaled(synth.CONFIGS[2], name=f"tiny_{P}_{G}_{T}_{H}_{V}", P=P, G=G, T=T, H=H, V=V, len_lo=0.5)
+    run_and_compare(trl, w)
+    run_and_compare(trl, w, fused=True)
+
+
 def test_minimum_workspace_gives_same_backward(trl):
     # chunked backward (one 128-row block per chunk) equals the one-chunk result
     w = synth.scaled(synth.CONFIGS[2], name="chunks", P=1, G=3, T=200, H=128, V=512)
