@@ -349,7 +349,7 @@ def main():
     host_out = torch.empty(5, dtype=torch.float32).pin_memory()
     h2d = sum(v.numel() * v.element_size() for v in host.values())
     d2h = host_out.numel() * 4
-    e2e_steps = max(2, min(args.steps, 4))
+    e2e_steps = max(2, min(args.steps, 8))
     sets = [batch, {**batch, **{k: torch.empty_like(batch[k]) for k in in_keys}}]
     copy_stream = torch.cuda.Stream()
     uploaded = [torch.cuda.Event(), torch.cuda.Event()]
