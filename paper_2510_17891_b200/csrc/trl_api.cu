@@ -10,7 +10,7 @@ namespace {
 constexpr int kRecommendedChunkRowsBf16 = 32768;
 constexpr int kRecommendedChunkRowsF32 = 2048;
 constexpr int kRasterBandFwd = 32;
-constexpr int kRasterBandFwdE = 24;   // forward tiles that also store E / dS
+constexpr int kRasterBandFwdE = 16;   // forward 256x256 tiles that also store E / dS (in CTA tiles)
 constexpr int kRasterBandBwd = 4;
 
 int check_device() {      // the current device must be compute capability 10.x (cached per device)

@@ -17,10 +17,10 @@
 //         so the forward GEMM is not repeated in the backward.
 //
 // Roles: warp 0 = TMA producer (one elected lane), warp 1 = MMA issuer (one elected lane)
-// and TMEM owner, warps 2..5 = epilogue (one TMEM lane quadrant each).  Shared-memory
+// and TMEM owner, warps 2.. = epilogue (groups of four warps, one TMEM lane quadrant each).  Shared-memory
 // stages are guarded by full/empty mbarriers; the 512 TMEM columns hold two 128x256 fp32
-// accumulators: in the forward GEMMs the epilogue of tile i overlaps the mainloop of tile
-// i+1, in the gradient GEMMs both belong to one 256x256 CTA tile that shares its B operand.
+// accumulators: in the scoring GEMM the epilogue of tile i overlaps the mainloop of tile
+// i+1, in the other GEMMs both belong to one 256x256 CTA tile that shares its B operand.
 // The dS / E / dW epilogues stage 32-row x 128-byte units in swizzled shared memory and hand
 // them to the TMA (bulk tensor store / reduce-add), so global memory sees whole 128 B lines.
 // Every wait is bounded: on expiry the CTA raises TRL_ERR_TIMEOUT in the status word,
@@ -37,7 +37,6 @@ constexpr int BM = 128, BN = 256, BK = 64, UMMA_K = 16, STAGES = 4;
 constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int OUT_STAGE_BYTES = 4 * 2 * 4096;   // 4 epilogue warps x 2 buffers x (32 rows x 128 B)
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + OUT_STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
-constexpr int NUM_THREADS = 192;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr float LOG2E = 1.4426950408889634f, LN2 = 0.6931471805599453f;
 constexpr long long WAIT_CYCLES = 4000000000LL;   // ~2-3 s at B200 clocks
@@ -183,16 +182,21 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 
 // Per-warp staged output: each lane owns one 128-byte row of a 32-row unit.  Rows are
 // written with the 128-byte swizzle (16-byte chunk index XOR row%8) the tensor map expects,
-// then one lane issues the bulk tensor store (or fp32 reduce-add); two buffers alternate.
+// then one lane issues the bulk tensor store (or fp32 reduce-add).  With 4 epilogue warps each
+// warp alternates between two 4 KB buffers, with 8 warps each has one.
 struct WarpOut {
-  uint32_t smem;            // this warp's two 4 KB buffers, 1024-byte aligned
+  uint32_t smem;            // this warp's 4 KB buffer(s), 1024-byte aligned
   const CUtensorMap* tm;
   int lane;
   int n;
+  int nbuf;                 // buffers in use: 2 (alternating) or 1
   template <bool REDUCE>
   __device__ __forceinline__ void put(const uint4 (&w)[8], int x, int y) {
-    const uint32_t buf = smem + (uint32_t)(n & 1) * 4096u;
-    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+    const uint32_t buf = smem + (uint32_t)(nbuf == 2 ? (n & 1) : 0) * 4096u;
+    if (lane == 0) {          // the store that last used this buffer must have read it
+      if (nbuf == 2) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+      else asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+    }
     __syncwarp();
     const uint32_t row = buf + (uint32_t)lane * 128u;
 #pragma unroll
@@ -376,24 +380,28 @@ __device__ __forceinline__ void epilogue_tile(const TcArgs& p, uint32_t tmem_acc
 }
 
 // ---------------------------------------------------------------- the kernel
-// MT = 128-row M blocks per CTA tile.  The forward GEMMs (K = H, short mainloop) use MT = 1 and
-// alternate between two TMEM accumulators so the epilogue overlaps the next mainloop.  The
-// gradient GEMMs (K = V or K = rows of a chunk: long mainloop, operands streaming from HBM)
+// MT = 128-row M blocks per CTA tile.  The scoring GEMM (LSE) uses MT = 1 and alternates
+// between two TMEM accumulators so the epilogue overlaps the next mainloop.  All other GEMMs
 // use MT = 2: one B tile in shared memory feeds both accumulators, which cuts the shared-memory
-// fill traffic per FLOP by a third; their epilogue is a few % of the mainloop and runs exposed.
+// fill traffic per FLOP by a third, and the epilogue runs exposed.  For the gradient GEMMs
+// (K = V or K = rows of a chunk) it is 0.4-2 % of the mainloop; for the forward GEMMs that
+// store dS / E (K = H) two epilogue warp groups drain the two accumulators at the same time.
 template <int EPI> struct TileCfg {
-  static constexpr int MT = (EPI == TC_EPI_DH || EPI == TC_EPI_DW) ? 2 : 1;
+  static constexpr int MT = (EPI == TC_EPI_LSE) ? 1 : 2;
+  // epilogue warp groups (4 warps each) working in parallel, one accumulator each
+  static constexpr int EG = (EPI == TC_EPI_E || EPI == TC_EPI_DS) ? 2 : 1;
+  static constexpr int THREADS = 64 + 128 * EG;
   static constexpr int NACC = 2 / MT;                       // accumulator sets in the 512 TMEM columns
   static constexpr int STG_BYTES = MT * A_BYTES + B_BYTES;  // 48 KB or 64 KB
   static constexpr int NSTAGE = (STAGES * STAGE_BYTES) / STG_BYTES;   // 4 or 3
 };
 
 template <int EPI>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+__global__ void __launch_bounds__(TileCfg<EPI>::THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmOut, const TcArgs p) {
   using Cfg = TileCfg<EPI>;
-  constexpr int MT = Cfg::MT, NACC = Cfg::NACC, NSTAGE = Cfg::NSTAGE, STG = Cfg::STG_BYTES;
+  constexpr int MT = Cfg::MT, NACC = Cfg::NACC, NSTAGE = Cfg::NSTAGE, STG = Cfg::STG_BYTES, EG = Cfg::EG;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t out_base = smem_base + STAGES * STAGE_BYTES;          // 1024-aligned
@@ -437,7 +445,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 128); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 128 * EG); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -546,9 +554,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
     __syncwarp();
   } else {
-    // ------------------------------------------------------------ epilogue warps 2..5
-    const int quad = warp & 3;
-    WarpOut wo{out_base + (uint32_t)quad * 8192u, &tmOut, lane, 0};
+    // ------------------------------------------------------------ epilogue warps: EG groups of 4
+    const int quad = warp & 3;           // TMEM lane quadrant this warp may read
+    const int grp = (warp - 2) / 4;      // group g drains the accumulators j with j % EG == g
+    WarpOut wo{out_base + (uint32_t)(warp - 2) * (8192u / EG), &tmOut, lane, 0, 2 / EG};
     int acc = 0; uint32_t acc_phase = 0;
     for (int tile = blockIdx.x; tile < total; tile += gridDim.x) {
       int ms, nt;
@@ -561,7 +570,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       tc_fence_after();
 #pragma unroll
       for (int j = 0; j < MT; ++j)
-        if (mask & (1 << j)) epilogue_tile<EPI>(p, tmem_base + (uint32_t)((acc * MT + j) * BN), quad, lane, ms * MT + j, nt, wo);
+        if ((mask & (1 << j)) && (j % EG) == grp) epilogue_tile<EPI>(p, tmem_base + (uint32_t)((acc * MT + j) * BN), quad, lane, ms * MT + j, nt, wo);
       tc_fence_before();
       mbar_arrive(tempty_bar(acc));
       if (++acc == NACC) { acc = 0; acc_phase ^= 1u; }
@@ -637,7 +646,7 @@ cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUt
     if (e != cudaSuccess) return e;
     attr_set[dev] = true;
   }
-  tc_gemm_kernel<EPI><<<grid, NUM_THREADS, SMEM_BYTES, s>>>(tmA, tmB, tmOut, a);
+  tc_gemm_kernel<EPI><<<grid, TileCfg<EPI>::THREADS, SMEM_BYTES, s>>>(tmA, tmB, tmOut, a);
   note_launch();
   return cudaGetLastError();
 }
@@ -672,7 +681,7 @@ cudaError_t launch_tc_gemm(const TcGemm& g, cudaStream_t s) {
   a.dHidden = g.dHidden; a.dh_ld = g.dh_ld; a.dW = g.dW; a.dw_ld = g.dw_ld; a.status = g.status;
   a.psum = g.psum; a.row_scale = g.row_scale; a.blk_active = g.blk_active;
   const int NT = cdiv(g.N, BN);
-  const int mt = (g.epi == TC_EPI_DW || g.epi == TC_EPI_DH) ? 2 : 1;
+  const int mt = (g.epi == TC_EPI_LSE) ? 1 : 2;
   const long max_tiles = (long)cdiv(g.epi == TC_EPI_DW ? g.m_blocks : g.blk_cap, mt) * NT;
   const int grid = (int)(max_tiles < (long)tc_num_sms() ? (max_tiles > 0 ? max_tiles : 1) : tc_num_sms());
   switch (g.epi) {
