@@ -90,3 +90,46 @@ def test_repeated_runs_are_bit_identical(trl):
     for a, c in ((runs[0], runs[1]), (runs[2], runs[3])):
         for k in a:
             assert torch.equal(a[k], c[k]), k
+
+
+def test_step_replays_from_a_cuda_graph(trl):
+    """The calls enqueue work on the caller's stream only (no allocation, no host sync), so a
+    whole step can be captured once and replayed with new input values in the same buffers."""
+    w = synth.scaled(synth.CONFIGS[2], name="graph", P=2, G=4, T=300, H=256, V=2048)
+    b = synth.make_batch(w, device=DEV)
+    B, T, H, V = w.B, w.T, w.H, w.V
+    f32 = dict(dtype=torch.float32, device=DEV)
+    ws = lambda call: torch.empty(trl.trl_workspace_bytes(call, B, T, H, V, trl.TRL_BF16), dtype=torch.uint8, device=DEV)
+    bufs = dict(old_logp=torch.empty(w.N, **f32), old_lse=torch.empty(w.N, **f32), ws_fwd=ws(trl.TRL_CALL_TOKEN_LOGPROBS),
+                ws_fused=ws(trl.TRL_CALL_PG_STEP_FUSED),
+                fused_out=dict(logp=torch.empty(w.N, **f32), lse=torch.empty(w.N, **f32), g=torch.empty(w.N, **f32),
+                               loss=torch.empty(1, **f32), stats=torch.empty(4, **f32),
+                               dHidden=torch.empty_like(b["hidden"]), dW=torch.empty(V, H, **f32)))
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    out = trl.hrd_pg_step(b, w.P, w.G, T, fused=True, bufs=bufs, status=status)       # eager (also warms up)
+    bufs["hrd"] = out["hrd"]
+    torch.cuda.synchronize()
+    eager = {k: out[k].clone() for k in ("logp", "loss", "dHidden", "dW")}
+    stream = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        with torch.cuda.graph(graph, stream=stream):
+            trl.hrd_pg_step(b, w.P, w.G, T, fused=True, bufs=bufs, status=status, stream=stream)
+    for k in ("logp", "loss", "dHidden", "dW"):
+        out[k].fill_(float("nan"))
+    graph.replay()
+    torch.cuda.synchronize()
+    for k in eager:
+        assert torch.equal(out[k], eager[k]), k
+    # new inputs in the same buffers: the replay follows them
+    b2 = synth.make_batch(synth.scaled(w, name="graph2"), device=DEV)
+    for k in ("hidden", "W", "W_old", "ids", "lens", "bnd", "r_plan", "r_code"):
+        b[k].copy_(b2[k])
+    graph.replay()
+    torch.cuda.synchronize()
+    replayed = {k: out[k].clone() for k in eager}
+    ref = trl.hrd_pg_step(b2, w.P, w.G, T, fused=True, status=status)
+    torch.cuda.synchronize()
+    trl.check_status(status)
+    for k in eager:
+        assert torch.equal(replayed[k], ref[k]), k
