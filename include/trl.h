@@ -25,10 +25,20 @@
  *  - Return value: TRL_OK or an error found on the host (bad argument, shape, workspace,
  *    CUDA launch error).  Errors found on the device (token id outside [0,V), len outside
  *    [0,T], bnd outside [0,len], a pipeline wait that ran out) are OR-ed as bit
- *    (1 << code) into *status_dev (int32, caller zero-initialises it; may be NULL).  Offending rows
- *    are treated as padding / clamped, so no out-of-bounds access happens.
+ *    (1 << code) into *status_dev (int32, caller zero-initialises it; may be NULL).  Lengths
+ *    and boundaries are clamped; a row whose token id is out of range gets logp = 0 from the call
+ *    that scores it and adds nothing to dHidden / dW (trl_pg_step_fused also leaves it out of
+ *    the loss and of g; trl_pg_loss_fwd never sees ids and evaluates it with logp = 0).  No
+ *    out-of-bounds access happens.
  *  - Outputs for padded rows (t >= len[b]) are defined: 0.
  *  - Row-major everywhere.  bf16 tensors need H % 8 == 0 and V % 8 == 0 (16-byte rows).
+ *  - Alignment.  Every [B*T] and every matrix argument (hidden, W, dHidden, dW, ids, logp,
+ *    old_logp, lse, adv, seg, g) must start on a 16-byte boundary: the kernels use 16-byte
+ *    accesses and TMA on them.  Per-rollout arrays and scalars (len, bnd, rewards, A_*, n_*,
+ *    loss, stats, status_dev) need the alignment of their element type (n_valid: 8 bytes).  A
+ *    call given a pointer that breaks this returns TRL_ERR_INVALID_ARG before anything is
+ *    launched.  (Allocations from cudaMalloc or a framework's allocator are 256-byte aligned;
+ *    the rule matters for offset views into them.)
  */
 #ifndef TRL_H_
 #define TRL_H_

@@ -61,11 +61,6 @@ def token_logprobs(hidden, W, ids, lens, T):
     return logp, lse
 
 
-def row_logits(hidden_row, W):
-    """z[v] = sum_k hidden_row[k] W[v,k] for one row (used for sampled-row checks)."""
-    return _f64(W) @ _f64(hidden_row)
-
-
 def hrd_advantages(r_plan, r_code, lens, bnd, P, G, T, adv_mode=0):
     """Hierarchical Reward Decomposition: segment labels and group-relative advantages.
 
@@ -231,6 +226,31 @@ def row_dhidden(hidden_row, W, tok, g_n):
     dS = -p
     dS[int(tok)] += 1.0
     return g_n * (dS @ W)
+
+
+def dW_rows(hidden, W_rows, vsel, ids, lens, lse, g, T):
+    """Selected rows of dW: dW[v] = sum_n g[n] (1[v = ids[n]] - exp(z[n,v] - lse[n])) hidden[n,:] for
+    v in `vsel`, summed over all valid rows n, with z[n,v] = hidden[n] . W_rows[k] for v = vsel[k]
+    (the same chain rule as pg_loss_bwd, restricted to a few vocabulary rows so that it can be
+    evaluated at full size).  `lse` and `g` are given per row.  Returns [len(vsel), H] float64."""
+    hidden = _f64(hidden)
+    W_rows = _f64(W_rows)
+    vsel = np.asarray(vsel, dtype=np.int64)
+    ids = np.asarray(ids, dtype=np.int64)
+    lens = np.asarray(lens, dtype=np.int64)
+    lse = _f64(lse)
+    g = _f64(g)
+    out = np.zeros((vsel.shape[0], hidden.shape[1]), dtype=np.float64)
+    for b in range(lens.shape[0]):
+        L = int(lens[b])
+        if L == 0:
+            continue
+        rows = slice(b * T, b * T + L)
+        z = hidden[rows] @ W_rows.T                                   # [L, len(vsel)]
+        dS = (ids[rows][:, None] == vsel[None, :]).astype(np.float64) - np.exp(z - lse[rows][:, None])
+        dS *= g[rows][:, None]
+        out += dS.T @ hidden[rows]
+    return out
 
 
 def full_step(hidden, W, hidden_old, W_old, ids, lens, bnd, r_plan, r_code, P, G, T,

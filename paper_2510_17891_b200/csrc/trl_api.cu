@@ -1,4 +1,5 @@
 // extern "C" entry points of libtrl: argument checks, workspace carving, kernel sequencing.
+#include <atomic>
 #include <cstring>
 
 #include "trl_internal.h"
@@ -14,16 +15,22 @@ constexpr int kRasterBandFwdE = 16;   // forward 256x256 tiles that also store E
 constexpr int kRasterBandBwd = 4;
 
 int check_device() {      // the current device must be compute capability 10.x (cached per device)
-  static int cached[64];
-  static bool known[64] = {};
+  static std::atomic<int> cached[64];      // 0: not looked up yet; otherwise status + 1
   int dev = 0, major = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return TRL_ERR_CUDA;
-  if (known[dev]) return cached[dev];
+  const int c = cached[dev].load(std::memory_order_relaxed);
+  if (c) return c - 1;
   if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return TRL_ERR_CUDA;
-  cached[dev] = (major == 10) ? TRL_OK : TRL_ERR_ARCH;
-  known[dev] = true;
-  return cached[dev];
+  const int st = (major == 10) ? TRL_OK : TRL_ERR_ARCH;
+  cached[dev].store(st + 1, std::memory_order_relaxed);
+  return st;
 }
+
+// Alignment contract of the boundary: tensors the kernels touch with 16-byte accesses or through
+// TMA must start on a 16-byte boundary; everything else on the boundary of its element type.
+bool al16(const void* p) { return ((uintptr_t)p & 15) == 0; }
+bool al4(const void* p) { return ((uintptr_t)p & 3) == 0; }
+bool al8(const void* p) { return ((uintptr_t)p & 7) == 0; }
 
 bool shapes_ok(int B, int T, int H, int V) {
   return B > 0 && T > 0 && H > 0 && V > 0 && (long)B * T < (1L << 31) - 256 && (long)V * H < (1L << 40);
@@ -147,6 +154,8 @@ int trl_token_logprobs(const void* hidden, const void* W, const int32_t* ids, co
   if (!shapes_ok(B, T, H, V)) return TRL_ERR_SHAPE;
   if (dt == TRL_BF16 && ((H % 8) || (V % 8))) return TRL_ERR_SHAPE;
   if (((uintptr_t)workspace & 255) != 0) return TRL_ERR_INVALID_ARG;
+  if (!al16(hidden) || !al16(W) || !al16(ids) || !al4(len) || !al16(logp) || !al16(lse) || (status_dev && !al4(status_dev)))
+    return TRL_ERR_INVALID_ARG;
   if (workspace_bytes < trl_workspace_bytes_min(TRL_CALL_TOKEN_LOGPROBS, B, T, H, V, dt)) return TRL_ERR_WORKSPACE_TOO_SMALL;
   if (int e = check_device()) return e;
   cudaStream_t s = (cudaStream_t)stream;
@@ -199,6 +208,9 @@ int trl_hrd_advantages(const float* r_plan, const float* r_code, const int32_t* 
     return TRL_ERR_INVALID_ARG;
   if (P <= 0 || G <= 0 || T <= 0 || (long)P * G > 65535 || (long)P * G * T >= (1L << 31)) return TRL_ERR_SHAPE;
   if (adv_mode != 0 && adv_mode != 1) return TRL_ERR_INVALID_ARG;
+  if (!al4(r_plan) || !al4(r_code) || !al4(len) || !al4(bnd) || !al4(A_plan) || !al4(A_code) || !al16(seg) || !al16(adv) ||
+      !al4(n_plan) || !al4(n_code) || !al8(n_valid) || (status_dev && !al4(status_dev)))
+    return TRL_ERR_INVALID_ARG;
   if (int e = check_device()) return e;
   launch_hrd_advantages(r_plan, r_code, len, bnd, P, G, T, adv_mode, A_plan, A_code, seg, adv, n_plan, n_code,
                         n_valid, status_dev, (cudaStream_t)stream);
@@ -214,9 +226,13 @@ int trl_pg_loss_fwd(const float* logp, const float* old_logp, const float* adv, 
   if (P <= 0 || G <= 0 || T <= 0 || (long)P * G > 65535 || (long)P * G * T >= (1L << 31)) return TRL_ERR_SHAPE;
   if (!(cfg.eps_lo >= 0.f) || !(cfg.eps_hi >= 0.f) || !(cfg.alpha >= 0.f) || (cfg.clip_form & ~1) || (cfg.agg_mode & ~1))
     return TRL_ERR_INVALID_ARG;
+  if (((uintptr_t)workspace & 255) != 0) return TRL_ERR_INVALID_ARG;
+  if (!al16(logp) || !al16(old_logp) || !al16(adv) || !al16(seg) || !al16(g) || !al4(len) || !al4(loss) || (stats && !al4(stats)))
+    return TRL_ERR_INVALID_ARG;
   if (workspace_bytes < trl_workspace_bytes(TRL_CALL_PG_LOSS_FWD, P * G, T, 1, 1, TRL_F32)) return TRL_ERR_WORKSPACE_TOO_SMALL;
   if (int e = check_device()) return e;
-  launch_pg_loss(logp, old_logp, adv, seg, len, P, G, T, cfg, loss, g, stats, (float*)workspace, (cudaStream_t)stream);
+  launch_pg_loss(logp, old_logp, adv, seg, len, P, G, T, cfg, loss, g, stats, (float*)workspace, nullptr, 0,
+                 (cudaStream_t)stream);
   TRL_CUDA_OK(cudaGetLastError());
   return TRL_OK;
 }
@@ -229,11 +245,24 @@ int trl_pg_loss_bwd(const void* hidden, const void* W, const int32_t* ids, const
   if (!shapes_ok(B, T, H, V)) return TRL_ERR_SHAPE;
   if (dt == TRL_BF16 && ((H % 8) || (V % 8))) return TRL_ERR_SHAPE;
   if (((uintptr_t)workspace & 255) != 0) return TRL_ERR_INVALID_ARG;
+  if (!al16(hidden) || !al16(W) || !al16(dHidden) || !al16(dW) || !al16(ids) || !al4(len) || !al16(lse) || !al16(g) ||
+      (status_dev && !al4(status_dev)))
+    return TRL_ERR_INVALID_ARG;
   if (workspace_bytes < trl_workspace_bytes_min(TRL_CALL_PG_LOSS_BWD, B, T, H, V, dt)) return TRL_ERR_WORKSPACE_TOO_SMALL;
   if (int e = check_device()) return e;
   cudaStream_t s = (cudaStream_t)stream;
   const int cap_rows = rows_cap_of(B, T);
   const size_t N = (size_t)B * T;
+  // rows per chunk that the workspace allows; decided before anything is enqueued
+  int R = 0;
+  if (dt == TRL_BF16) {
+    R = fit_rows(workspace_bytes - bwd_fixed_bf16(B, T, H, V), cap_rows < kRecommendedChunkRowsBf16 ? cap_rows : kRecommendedChunkRowsBf16,
+                 [&](int r) { return bwd_per_rows_bf16(H, V, r); });
+  } else {
+    R = fit_rows(workspace_bytes - row_pack_bytes(B, T), cap_rows < kRecommendedChunkRowsF32 ? cap_rows : kRecommendedChunkRowsF32,
+                 [&](int r) { return 2 * align_up((size_t)r * H * 4, 256) + align_up((size_t)r * V * 4, 256); });
+  }
+  if (R < kRowBlock) return TRL_ERR_WORKSPACE_TOO_SMALL;
 
   Carver cv(workspace);
   RowPack rb = carve_row_pack(cv.take<char>(row_pack_bytes(B, T)), B, T);
@@ -242,10 +271,6 @@ int trl_pg_loss_bwd(const void* hidden, const void* W, const int32_t* ids, const
 
   if (dt == TRL_BF16) {
     TRL_CUDA_OK(cudaMemsetAsync(dHidden, 0, N * H * 2, s));
-    const size_t avail = workspace_bytes - bwd_fixed_bf16(B, T, H, V);
-    const int R = fit_rows(avail, cap_rows < kRecommendedChunkRowsBf16 ? cap_rows : kRecommendedChunkRowsBf16,
-                           [&](int r) { return bwd_per_rows_bf16(H, V, r); });
-    if (R < kRowBlock) return TRL_ERR_WORKSPACE_TOO_SMALL;
     __nv_bfloat16* Xp = cv.take<__nv_bfloat16>((size_t)cap_rows * H);
     int* blk_active = cv.take<int>(rb.cap);
     __nv_bfloat16* dS = cv.take<__nv_bfloat16>((size_t)R * V);
@@ -279,10 +304,6 @@ int trl_pg_loss_bwd(const void* hidden, const void* W, const int32_t* ids, const
     }
   } else {
     TRL_CUDA_OK(cudaMemsetAsync(dHidden, 0, N * H * 4, s));
-    const size_t avail = workspace_bytes - row_pack_bytes(B, T);
-    const int R = fit_rows(avail, cap_rows < kRecommendedChunkRowsF32 ? cap_rows : kRecommendedChunkRowsF32,
-                           [&](int r) { return 2 * align_up((size_t)r * H * 4, 256) + align_up((size_t)r * V * 4, 256); });
-    if (R < kRowBlock) return TRL_ERR_WORKSPACE_TOO_SMALL;
     float* Xp = cv.take<float>((size_t)R * H);
     float* dHp = cv.take<float>((size_t)R * H);
     float* S = cv.take<float>((size_t)R * V);
@@ -320,6 +341,10 @@ int trl_pg_step_fused(const void* hidden, const void* W, const int32_t* ids, con
   if (!(cfg.eps_lo >= 0.f) || !(cfg.eps_hi >= 0.f) || !(cfg.alpha >= 0.f) || (cfg.clip_form & ~1) || (cfg.agg_mode & ~1))
     return TRL_ERR_INVALID_ARG;
   if (((uintptr_t)workspace & 255) != 0) return TRL_ERR_INVALID_ARG;
+  if (!al16(hidden) || !al16(W) || !al16(dHidden) || !al16(dW) || !al16(ids) || !al4(len) || !al16(old_logp) || !al16(adv) ||
+      !al16(seg) || !al16(logp) || !al16(lse) || !al16(g) || !al4(loss) || (lse_hint && !al16(lse_hint)) || (stats && !al4(stats)) ||
+      (status_dev && !al4(status_dev)))
+    return TRL_ERR_INVALID_ARG;
   if (workspace_bytes < trl_workspace_bytes_min(TRL_CALL_PG_STEP_FUSED, B, T, H, V, dt)) return TRL_ERR_WORKSPACE_TOO_SMALL;
   if (int e = check_device()) return e;
 
@@ -402,8 +427,9 @@ int trl_pg_step_fused(const void* hidden, const void* W, const int32_t* ids, con
     dw.m_blocks = cdiv(V, kRowBlock); dw.dW = dW; dw.dw_ld = H; dw.V = V; dw.blk_active = blk_active;
     TRL_CUDA_OK(launch_tc_gemm(dw, s));
   }
-  // loss, statistics (and g once more, identically) over all rows now that logp is complete
-  launch_pg_loss(logp, old_logp, adv, seg, len, P, G, T, cfg, loss, g, stats, loss_partials, s);
+  // loss, statistics (and g once more, identically) over all rows now that logp is complete; rows
+  // whose token id is out of range stay out of it, as they stayed out of the gradients
+  launch_pg_loss(logp, old_logp, adv, seg, len, P, G, T, cfg, loss, g, stats, loss_partials, ids, V, s);
   TRL_CUDA_OK(cudaGetLastError());
   return TRL_OK;
 }

@@ -38,9 +38,10 @@ void launch_hrd_advantages(const float* r_plan, const float* r_code, const int32
                            float* adv, int32_t* n_plan, int32_t* n_code, int64_t* n_valid, int32_t* status,
                            cudaStream_t s);
 int  pg_loss_tiles(int T);
+// ids may be null; when given, tokens whose id is outside [0, V) are left out like padding
 void launch_pg_loss(const float* logp, const float* old_logp, const float* adv, const uint8_t* seg,
                     const int32_t* len, int P, int G, int T, trl_pg_config cfg, float* loss, float* g,
-                    float* stats, float* partials, cudaStream_t s);
+                    float* stats, float* partials, const int32_t* ids, int V, cudaStream_t s);
 // merge per-vocabulary-tile (max, sumexp) partials into lse / logp and scatter to global rows
 void launch_merge_lse(const float2* partials, const float* tgt, int n_tiles, int rows_cap, RowPack rb,
                       const int32_t* ids, const int32_t* len, int B, int T, int V, float* logp, float* lse,

@@ -47,6 +47,9 @@ extern "C" int trl_pg_loss_fwd_static(const float* logp, const float* old_logp, 
   if (P <= 0 || G <= 0 || T <= 0 || (long)P * G > 65535 || (long)P * G * T >= (1L << 31)) return TRL_ERR_SHAPE;
   if (!(cfg.eps_lo >= 0.f) || !(cfg.eps_hi >= 0.f) || !(cfg.alpha >= 0.f) || (cfg.clip_form & ~1) || (cfg.agg_mode & ~1))
     return TRL_ERR_INVALID_ARG;
+  if ((((uintptr_t)logp | (uintptr_t)old_logp | (uintptr_t)adv | (uintptr_t)seg | (uintptr_t)g) & 15) != 0 ||
+      (((uintptr_t)len | (uintptr_t)loss | (uintptr_t)stats) & 3) != 0)
+    return TRL_ERR_INVALID_ARG;          // same alignment contract as trl_pg_loss_fwd
   // size limit of the built-in scratch: P*G*ceil(T/16384) slots
   if ((long)P * G * trl::pg_loss_tiles(T) > kStaticLossSlots) return TRL_ERR_WORKSPACE_TOO_SMALL;
   int major = 0, dev = 0;
@@ -58,6 +61,7 @@ extern "C" int trl_pg_loss_fwd_static(const float* logp, const float* old_logp, 
   if (int e = partials_for_current_device(&partials)) return e;
   // Every slot the second kernel reads is written by the first one in this same call, so
   // nothing left over from an earlier call is ever read and nothing needs clearing.
-  trl::launch_pg_loss(logp, old_logp, adv, seg, len, P, G, T, cfg, loss, g, stats, partials, (cudaStream_t)stream);
+  trl::launch_pg_loss(logp, old_logp, adv, seg, len, P, G, T, cfg, loss, g, stats, partials, nullptr, 0,
+                      (cudaStream_t)stream);
   return cudaGetLastError() == cudaSuccess ? TRL_OK : TRL_ERR_CUDA;
 }

@@ -233,7 +233,8 @@ __device__ __forceinline__ long long total_valid_tokens(const int32_t* len, int 
 __global__ void __launch_bounds__(256) pg_loss_stage1_kernel(
     const float* __restrict__ logp, const float* __restrict__ old_logp, const float* __restrict__ adv,
     const uint8_t* __restrict__ seg, const int32_t* __restrict__ len, int P, int G, int T, trl_pg_config cfg,
-    float* __restrict__ g, float* __restrict__ partials) {
+    float* __restrict__ g, float* __restrict__ partials, const int32_t* __restrict__ ids, int V) {
+  // ids (may be null): tokens whose id is outside [0, V) are skipped like padding
   const int b = blockIdx.y, tid = threadIdx.x;
   const int L = max(0, min(len[b], T));
   const int t_begin = blockIdx.x * kLossTile, t_end = min(T, t_begin + kLossTile);
@@ -257,9 +258,12 @@ __global__ void __launch_bounds__(256) pg_loss_stage1_kernel(
         const uchar4 sg = *reinterpret_cast<const uchar4*>(seg + n);
         const float lpa[4] = {lp.x, lp.y, lp.z, lp.w}, ola[4] = {ol.x, ol.y, ol.z, ol.w}, ada[4] = {ad.x, ad.y, ad.z, ad.w};
         const int sga[4] = {sg.x, sg.y, sg.z, sg.w};
+        int4 idq = make_int4(0, 0, 0, 0);
+        if (ids) idq = *reinterpret_cast<const int4*>(ids + n);
+        const int ida[4] = {idq.x, idq.y, idq.z, idq.w};
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
-          if (t + k < L) {
+          if (t + k < L && (!ids || (unsigned)ida[k] < (unsigned)V)) {
             const TokenTerm tt = surrogate_token(lpa[k], ola[k], ada[k], sga[k], cfg, inv);
             acc += tt.wu;
             gq[k] = tt.g;
@@ -274,7 +278,7 @@ __global__ void __launch_bounds__(256) pg_loss_stage1_kernel(
   } else {
     for (int t = t_begin + tid; t < t_end; t += 256) {
       float gn = 0.f;
-      if (t < L) {
+      if (t < L && (!ids || (unsigned)ids[base + t] < (unsigned)V)) {
         const size_t n = base + t;
         const TokenTerm tt = surrogate_token(logp[n], old_logp[n], adv[n], seg[n], cfg, inv);
         acc += tt.wu;
@@ -343,10 +347,10 @@ __global__ void __launch_bounds__(256) pg_loss_stage2_kernel(const float* __rest
 
 void launch_pg_loss(const float* logp, const float* old_logp, const float* adv, const uint8_t* seg,
                     const int32_t* len, int P, int G, int T, trl_pg_config cfg, float* loss, float* g,
-                    float* stats, float* partials, cudaStream_t s) {
+                    float* stats, float* partials, const int32_t* ids, int V, cudaStream_t s) {
   const int tiles = pg_loss_tiles(T);
   dim3 grid(tiles, P * G);
-  pg_loss_stage1_kernel<<<grid, 256, 0, s>>>(logp, old_logp, adv, seg, len, P, G, T, cfg, g, partials);
+  pg_loss_stage1_kernel<<<grid, 256, 0, s>>>(logp, old_logp, adv, seg, len, P, G, T, cfg, g, partials, ids, V);
   note_launch();
   pg_loss_stage2_kernel<<<1, 256, 0, s>>>(partials, len, P, G, T, tiles, cfg.agg_mode, loss, stats);
   note_launch();
@@ -436,11 +440,15 @@ void launch_pack_rows_bf16(const __nv_bfloat16* src, __nv_bfloat16* out, int H, 
 }
 
 // ------------------------------------------------------------------------------------
-// Fused step, per chunk: one thread per scratch row.  With E = exp(z - c) stored by the GEMM,
-//   lse = c + log sum_v E,  logp = z[id] - lse,  g = d loss / d logp (same formula as
+// Fused step, per chunk: one thread per scratch row.  The GEMM stored E = exp(z - c), the sampled
+// token's logit z_t, and per vocabulary tile the row sum of E over every column except the sampled
+// token's.  With S' = sum_{v != t} E_v and E_t = exp(z_t - c):
+//   lse = c + log(S' + E_t),  logp = z_t - lse,  g = d loss / d logp (same formula as
 //   pg_loss_stage1_kernel),  dS = g onehot - g exp(c - lse) E = neg_alpha (E - exp(lse - c) onehot),
-// so the kernel stores neg_alpha = -g exp(c - lse) and subtracts exp(lse - c) from the
-// sampled token's entry of E.
+// so the kernel stores neg_alpha = -g exp(c - lse) and replaces the sampled token's entry of E by
+// E_t - exp(lse - c) = -S'.  Formed this way the entry has no cancellation however close the
+// token's probability is to 1 (E_t and exp(lse - c) then agree to many digits).
+// A row whose token id is out of range is flagged and treated as padding (g = 0).
 // ------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(128) fused_merge_kernel(FusedMergeArgs a) {
   // one CTA = one 128-row block of the chunk
@@ -451,15 +459,17 @@ __global__ void __launch_bounds__(128) fused_merge_kernel(FusedMergeArgs a) {
   if (r < a.R && q < a.rb.n_rows[0]) {
     const size_t n = (size_t)a.rb.rowmap[q];
     const int b = (int)(n / a.T);
-    float sum = 0.f;
-    for (int k = 0; k < a.n_tiles; ++k) sum += a.psum[(size_t)k * a.R + r];
+    float s_excl = 0.f;
+    for (int k = 0; k < a.n_tiles; ++k) s_excl += a.psum[(size_t)k * a.R + r];
     const float c = a.hint[n];
-    const float lse = c + logf(sum);
     const int id = a.ids[n];
     const bool id_ok = (unsigned)id < (unsigned)a.V;
     if (!id_ok) flag_status(a.status, TRL_ERR_BAD_INDEX);
+    const float zt = id_ok ? a.tgt[r] : 0.f;
+    const float sum = s_excl + (id_ok ? expf(zt - c) : 0.f);
     if (!(sum > 0.f) || !isfinite(sum)) flag_status(a.status, TRL_ERR_BAD_HINT);
-    const float lp = id_ok ? a.tgt[r] - lse : 0.f;
+    const float lse = c + logf(sum);
+    const float lp = id_ok ? zt - lse : 0.f;
     a.logp[n] = lp;
     a.lse[n] = lse;
     const int L = max(0, min(a.len[b], a.T));
@@ -467,11 +477,7 @@ __global__ void __launch_bounds__(128) fused_merge_kernel(FusedMergeArgs a) {
     const TokenTerm tt = surrogate_token(lp, a.old_logp[n], a.adv[n], a.seg[n], a.cfg, inv);
     gn = id_ok ? tt.g : 0.f;
     a.g[n] = gn;
-    if (gn != 0.f) {
-      const float beta = expf(lse - c);
-      __nv_bfloat16* e = a.E + (size_t)r * a.V + id;
-      *e = __float2bfloat16_rn(__bfloat162float(*e) - beta);
-    }
+    if (gn != 0.f) a.E[(size_t)r * a.V + id] = __float2bfloat16_rn(-s_excl);
     gn = -gn * expf(c - lse);
   }
   if (r < a.R) a.neg_alpha[r] = gn;
@@ -570,8 +576,8 @@ __global__ void __launch_bounds__(256) ds_inplace_f32_kernel(float* __restrict__
     for (int v = threadIdx.x; v < V; v += 256) row[v] = 0.f;
     return;
   }
-  const float gn = g[n], L = lse[n];
   const int id = ids[n];
+  const float gn = (unsigned)id < (unsigned)V ? g[n] : 0.f, L = lse[n];     // a row with a bad id adds nothing
   for (int v = threadIdx.x; v < V; v += 256) row[v] = gn * ((v == id ? 1.f : 0.f) - expf(row[v] - L));
 }
 void launch_ds_inplace_f32(float* S, int V, int R, RowPack rb, int blk_off, const int32_t* ids, const float* lse,

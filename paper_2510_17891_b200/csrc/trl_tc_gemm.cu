@@ -12,7 +12,7 @@
 //   DH  : dHidden rows (bf16), scattered to the caller's row positions
 //   DW  : dW += tile (fp32, TMA reduce-add from shared memory)
 //   E   : E = exp(z - c) for a per-row shift c (a stale log-partition), as bf16, plus the row
-//         sums of E and the sampled token's logit.  The softmax is p = E exp(c - lse), a
+//         sums of E over every column but the sampled token's, and the sampled token's logit.  The softmax is p = E exp(c - lse), a
 //         per-row factor the gradient GEMMs fold into their other operand / their epilogue,
 //         so the forward GEMM is not repeated in the backward.
 //
@@ -26,6 +26,8 @@
 // Every wait is bounded: on expiry the CTA raises TRL_ERR_TIMEOUT in the status word,
 // all roles leave their loops, TMEM is freed and the kernel returns.
 #include <cuda.h>
+
+#include <atomic>
 
 #include "trl_internal.h"
 
@@ -280,7 +282,7 @@ __device__ __forceinline__ void epilogue_tile(const TcArgs& p, uint32_t tmem_acc
     const int id = valid ? p.ids[grow] : -1;
     const float gg = valid ? p.g[grow] : 0.f;
     const float L2 = valid ? p.lse[grow] * LOG2E : 0.f;
-    const bool live = valid && gg != 0.f;
+    const bool live = valid && gg != 0.f && (unsigned)id < (unsigned)p.N;   // a row with a bad id adds nothing
     for (int c0 = 0; c0 < BN; c0 += 64) {
       if (p.N - (n0 + c0) <= 0) break;
       uint4 w[8];
@@ -320,18 +322,23 @@ __device__ __forceinline__ void epilogue_tile(const TcArgs& p, uint32_t tmem_acc
         tc_ld32(taddr + c0 + 32 * h, v);
         tc_wait_ld();
         float d[32];
+        float gs = 0.f;
 #pragma unroll
         for (int j = 0; j < 32; ++j) {
           const float e = ex2(fmaf(__uint_as_float(v[j]), LOG2E, -C2));
           d[j] = (valid && j < ncl) ? e : 0.f;
-          sum += d[j];
+          gs += d[j];
         }
         const int lc = id - (n0 + c0 + 32 * h);
-        if (lc >= 0 && lc < 32 && lc < ncl) {
+        if (lc >= 0 && lc < 32 && lc < ncl) {      // the sampled token's column: keep it out of the row sum
+          gs = 0.f;
 #pragma unroll
-          for (int j = 0; j < 32; ++j) if (j == lc) tg = __uint_as_float(v[j]);
+          for (int j = 0; j < 32; ++j) {
+            if (j == lc) tg = __uint_as_float(v[j]); else gs += d[j];
+          }
           has = true;
         }
+        sum += gs;
 #pragma unroll
         for (int q = 0; q < 4; ++q)
           w[4 * h + q] = make_uint4(pack_bf16x2(d[q * 8 + 0], d[q * 8 + 1]), pack_bf16x2(d[q * 8 + 2], d[q * 8 + 3]),
@@ -592,15 +599,16 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
+EncodeTiledFn lookup_encode_fn() {
+  void* ptr = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+      qres == cudaDriverEntryPointSuccess)
+    return (EncodeTiledFn)ptr;
+  return nullptr;
+}
 EncodeTiledFn get_encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  if (!fn) {
-    void* ptr = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
-        qres == cudaDriverEntryPointSuccess)
-      fn = (EncodeTiledFn)ptr;
-  }
+  static const EncodeTiledFn fn = lookup_encode_fn();   // initialised once, also under concurrent first calls
   return fn;
 }
 
@@ -637,14 +645,14 @@ bool make_out_tmap(CUtensorMap* tm, void* base, long inner, long outer, long ld,
 template <int EPI>
 cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmOut, const TcArgs& a, int grid,
                        cudaStream_t s) {
-  static bool attr_set[64] = {};          // the attribute is per device
+  static std::atomic<bool> attr_set[64];   // the attribute is per device; setting it twice is harmless
   int dev = 0;
   cudaGetDevice(&dev);
   if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-  if (!attr_set[dev]) {
+  if (!attr_set[dev].load(std::memory_order_acquire)) {
     cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (e != cudaSuccess) return e;
-    attr_set[dev] = true;
+    attr_set[dev].store(true, std::memory_order_release);
   }
   tc_gemm_kernel<EPI><<<grid, TileCfg<EPI>::THREADS, SMEM_BYTES, s>>>(tmA, tmB, tmOut, a);
   note_launch();
@@ -654,12 +662,16 @@ cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUt
 }  // namespace
 
 int tc_num_sms() {
-  static int n[64] = {};
+  static std::atomic<int> n[64];
   int dev = 0;
   cudaGetDevice(&dev);
   if (dev < 0 || dev >= 64) return 1;
-  if (!n[dev]) cudaDeviceGetAttribute(&n[dev], cudaDevAttrMultiProcessorCount, dev);
-  return n[dev];
+  int v = n[dev].load(std::memory_order_relaxed);
+  if (!v) {
+    cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev);
+    n[dev].store(v, std::memory_order_relaxed);
+  }
+  return v > 0 ? v : 1;
 }
 
 cudaError_t launch_tc_gemm(const TcGemm& g, cudaStream_t s) {

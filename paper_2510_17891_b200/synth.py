@@ -14,6 +14,12 @@ Bernoulli(p_code) (optionally a fraction of prompts gets all-equal rewards);
 the old policy pi_theta_old shares the hidden states and has a perturbed LM head,
 W_old = W + sigma*N(0,1/H), which makes every logit differ by ~N(0, sigma) and hence the
 log-prob differences ~N(0, sigma), sigma = 0.05.
+
+Two generator-only knobs move the batch from this flat regime (no token above p ~ 1e-3) to the
+peaked one of a trained policy, where most sampled tokens carry almost all the probability:
+`logit_scale` multiplies the LM head (logits ~ N(0, logit_scale^2); the old policy's
+perturbation is not scaled, so log-prob differences stay ~N(0, sigma)), and `greedy_ids`
+takes ids = argmax of the logits instead of sampling.
 """
 from dataclasses import dataclass, replace
 import zlib
@@ -42,6 +48,8 @@ class Workload:
     degenerate_frac: float = 0.0  # fraction of prompts whose rewards are all equal
     real_plan_reward: bool = False  # plan reward Bernoulli * U(0.2, 2): the clipped speedup range
     sigma_old: float = 0.05
+    logit_scale: float = 1.0      # W ~ N(0, logit_scale^2 / H): larger = more confident policy
+    greedy_ids: bool = False      # ids = argmax of the logits instead of a sample from their softmax
 
     @property
     def B(self):
@@ -62,8 +70,6 @@ CONFIGS = {
                 len_lo=0.125, bnd_lo=0.5, bnd_hi=0.9),
     # one representative point of the config-4 sweep (the full grid is sweep_workloads())
     4: Workload("cfg4_V151936_H4096_G8", P=8, G=8, T=1024, H=4096, V=151936, degenerate_frac=0.25),
-    # not one of the five: a few-GB case of the same kernels for profiler captures
-    5: Workload("profile_small", P=1, G=8, T=2048, H=4096, V=32768),
 }
 
 
@@ -94,19 +100,22 @@ def _store_dtype(w: Workload):
     return torch.bfloat16 if w.dtype == "bf16" else torch.float32
 
 
-def sample_ids(hidden, W, gen, chunk_rows=2048):
-    """ids[n] ~ Categorical(softmax(hidden[n] W^T)) by Gumbel-max, in row chunks."""
+def sample_ids(hidden, W, gen, chunk_rows=2048, greedy=False):
+    """ids[n] ~ Categorical(softmax(hidden[n] W^T)) by Gumbel-max, in row chunks (greedy: the
+    argmax itself)."""
     N = hidden.shape[0]
     ids = torch.empty(N, dtype=torch.int32, device=hidden.device)
     mm_dtype = hidden.dtype if hidden.is_cuda else torch.float32
     Wm = W.to(mm_dtype)
     for r0 in range(0, N, chunk_rows):
         z = (hidden[r0:r0 + chunk_rows].to(mm_dtype) @ Wm.T).float()
-        u = torch.rand(z.shape, generator=gen, device=z.device, dtype=torch.float32)
-        u = u.clamp_(1e-20, 1.0 - 1e-7)
-        z.sub_(torch.log(-torch.log(u)))
+        if not greedy:
+            u = torch.rand(z.shape, generator=gen, device=z.device, dtype=torch.float32)
+            u = u.clamp_(1e-20, 1.0 - 1e-7)
+            z.sub_(torch.log(-torch.log(u)))
+            del u
         ids[r0:r0 + chunk_rows] = z.argmax(dim=1).to(torch.int32)
-        del z, u
+        del z
     return ids
 
 
@@ -125,7 +134,7 @@ def make_batch(w: Workload, device="cpu", seed_offset=0, with_old_model=True):
     hidden = torch.randn(N, H, generator=_gen(w, "hidden", dev, seed_offset), device=dev,
                          dtype=torch.float32).to(dt)
     W32 = torch.randn(V, H, generator=_gen(w, "W", dev, seed_offset), device=dev,
-                      dtype=torch.float32).mul_(H ** -0.5)
+                      dtype=torch.float32).mul_(w.logit_scale * H ** -0.5)
     W = W32.to(dt)
     out = dict(hidden=hidden, W=W)
     if with_old_model:
@@ -136,7 +145,7 @@ def make_batch(w: Workload, device="cpu", seed_offset=0, with_old_model=True):
         del dW
     del W32
 
-    out["ids"] = sample_ids(hidden, W, _gen(w, "ids", dev, seed_offset))
+    out["ids"] = sample_ids(hidden, W, _gen(w, "ids", dev, seed_offset), greedy=w.greedy_ids)
 
     gc = _gen(w, "lens", torch.device("cpu"), seed_offset)
     lo, hi = int(w.len_lo * T), int(w.len_hi * T)

@@ -60,3 +60,68 @@ def test_missing_library_fails_loudly(monkeypatch):
     monkeypatch.setattr(binding, "lib_path", lambda: "/nonexistent/libtrl.so")
     with pytest.raises(binding.TrlError):
         binding.load_library()
+
+
+def test_misaligned_pointers_are_rejected_on_the_host_before_any_launch():
+    """Every tensor the kernels touch with 16-byte accesses or TMA must be 16-byte aligned.  The
+    pointers below are never dereferenced: a misaligned one must make the call return
+    TRL_ERR_INVALID_ARG from its host-side checks, and the same call with aligned pointers but a
+    zero-byte workspace must get past those checks and stop at TRL_ERR_WORKSPACE_TOO_SMALL."""
+    import ctypes as C
+    import paper_2510_17891_b200 as trl
+    from paper_2510_17891_b200.binding import PgConfig
+    lib = trl.load_library()
+    base = 0x7f0000000000
+    A = lambda k: C.c_void_p(base + 0x100000 * k)            # distinct, 256-byte aligned
+    cfg = PgConfig(0.2, 0.2, 0.1, 0, 0)
+    B, T, H, V, P, G = 4, 64, 64, 512, 2, 2
+    INVALID, TOO_SMALL = 1, 4
+
+    def logprobs(off=(), ws_bytes=0):
+        a = [A(k) if k not in off else C.c_void_p(base + 0x100000 * k + 4) for k in range(8)]
+        return lib.trl_token_logprobs(a[0], a[1], a[2], a[3], B, T, H, V, trl.TRL_BF16, a[4], a[5], a[6], ws_bytes, None, None)
+
+    assert logprobs() == TOO_SMALL
+    for k in (0, 1, 2, 4, 5):                                 # hidden, W, ids, logp, lse
+        assert logprobs(off=(k,)) == INVALID, k
+    assert logprobs(off=(6,), ws_bytes=1 << 40) == INVALID    # workspace
+
+    def loss_fwd(off=(), ws_bytes=0):
+        a = [A(k) if k not in off else C.c_void_p(base + 0x100000 * k + 4) for k in range(10)]
+        return lib.trl_pg_loss_fwd(a[0], a[1], a[2], a[3], a[4], P, G, T, cfg, a[5], a[6], a[7], a[8], ws_bytes, None, None)
+
+    assert loss_fwd() == TOO_SMALL
+    for k in (0, 1, 2, 3, 6):                                 # logp, old_logp, adv, seg, g
+        assert loss_fwd(off=(k,)) == INVALID, k
+    assert loss_fwd(off=(8,), ws_bytes=1 << 30) == INVALID    # workspace (was unchecked before)
+
+    def loss_bwd(off=(), ws_bytes=0):
+        a = [A(k) if k not in off else C.c_void_p(base + 0x100000 * k + 4) for k in range(10)]
+        return lib.trl_pg_loss_bwd(a[0], a[1], a[2], a[3], a[4], a[5], B, T, H, V, trl.TRL_BF16, a[6], a[7], a[8], ws_bytes, None, None)
+
+    assert loss_bwd() == TOO_SMALL
+    for k in (0, 1, 2, 4, 5, 6, 7):                           # hidden, W, ids, lse, g, dHidden, dW
+        assert loss_bwd(off=(k,)) == INVALID, k
+
+    def fused(off=(), ws_bytes=0):
+        a = [A(k) if k not in off else C.c_void_p(base + 0x100000 * k + 4) for k in range(17)]
+        return lib.trl_pg_step_fused(a[0], a[1], a[2], a[3], a[4], a[5], a[6], a[7], P, G, T, H, V, trl.TRL_BF16, cfg,
+                                     a[8], a[9], a[10], a[11], a[12], a[13], a[14], a[15], ws_bytes, None, None)
+
+    assert fused() == TOO_SMALL
+    for k in (0, 1, 2, 4, 5, 6, 7, 8, 9, 11, 13, 14):         # every [B*T] and matrix argument
+        assert fused(off=(k,)) == INVALID, k
+
+    def hrd(off=()):
+        a = [A(k) if k not in off else C.c_void_p(base + 0x100000 * k + 4) for k in range(11)]
+        return lib.trl_hrd_advantages(a[0], a[1], a[2], a[3], P, G, T, 0, a[4], a[5], a[6], a[7], a[8], a[9], a[10], None, None)
+
+    for k in (6, 7, 10):                                      # seg, adv (16 bytes), n_valid (8 bytes)
+        assert hrd(off=(k,)) == INVALID, k
+
+    def static(off=()):
+        a = [A(k) if k not in off else C.c_void_p(base + 0x100000 * k + 4) for k in range(8)]
+        return lib.trl_pg_loss_fwd_static(a[0], a[1], a[2], a[3], a[4], P, G, T, cfg, a[5], a[6], a[7], None, None)
+
+    for k in (0, 1, 2, 3, 6):
+        assert static(off=(k,)) == INVALID, k

@@ -154,6 +154,24 @@ def test_config2_whole_step_sampled_rows_and_invariants(trl, cfg2_batch, fused):
     assert float(col.abs().max()) <= 1e-2 * float(out["dW"].double().abs().sum(dim=0).max())
     assert torch.isfinite(out["dW"]).all() and torch.isfinite(out["loss"]).all()
 
+    # dW with the real (dense) g: a few hundred vocabulary rows against the oracle's sum over ALL
+    # valid rows.  The oracle takes lse[n] and g[n] from the GPU arrays; those are pinned by the
+    # sampled-row checks above (lse through logp, g directly), so what this adds is the dense
+    # accumulation over every row block and chunk.
+    r = np.random.default_rng(11)
+    vidx = valid.nonzero().squeeze(1)
+    ids_c = ids[vidx.cpu().numpy()]
+    top = np.argsort(np.bincount(ids_c, minlength=w.V))[::-1][:96]
+    vsel = np.unique(np.concatenate([top, [0, 127, 128, 255, 256, 383, w.V - 129, w.V - 128, w.V - 127, w.V - 1],
+                                     r.integers(w.V - 128, w.V, 24), r.integers(0, w.V, 160)]))
+    assert vsel.size >= 256
+    ref_rows = orc.dW_rows(f64(batch["hidden"][vidx]), W64[vsel], vsel, ids_c, np.array([ids_c.size]),
+                           f64(out["lse"][vidx]), f64(out["g"][vidx]), T=ids_c.size)
+    got_rows = f64(out["dW"][torch.as_tensor(vsel, device=DEV)])
+    assert rel_fro(got_rows, ref_rows) <= TOL_GRAD
+    row_err = np.linalg.norm(got_rows - ref_rows, axis=1) / np.linalg.norm(ref_rows, axis=1)
+    assert row_err.max() <= 2 * TOL_GRAD, (row_err.max(), int(vsel[np.argmax(row_err)]))
+
 
 def test_full_size_advantages_and_loss_all_tokens(trl):
     """Steps a3 and a4 at the largest token count (config 3: 32 x 8192), every element
@@ -187,13 +205,14 @@ def test_full_size_advantages_and_loss_all_tokens(trl):
     np.testing.assert_allclose(f64(stats), rs, rtol=1e-4, atol=1e-6)
 
 
-def test_config3_long_reasoning_whole_step(trl):
-    """Config 3 (32 rollouts x 8192 tokens, heavy padding skew): whole step, sampled rows."""
+@pytest.mark.parametrize("fused", [False, True])
+def test_config3_long_reasoning_whole_step(trl, fused):
+    """Config 3 (32 rollouts x 8192 tokens, heavy padding skew): whole step on both schedules, sampled rows."""
     w = synth.CONFIGS[3]
     batch = synth.make_batch(w, device=DEV)
     lens, bnd, ids = batch["lens"].cpu().numpy(), batch["bnd"].cpu().numpy(), batch["ids"].cpu().numpy()
     status = torch.zeros(1, dtype=torch.int32, device=DEV)
-    out = trl.hrd_pg_step(batch, w.P, w.G, w.T, status=status)
+    out = trl.hrd_pg_step(batch, w.P, w.G, w.T, status=status, fused=fused)
     torch.cuda.synchronize()
     trl.check_status(status)
     rows = sample_rows(w, lens, bnd, n_random=16, n_rollouts=6, seed=5)
@@ -213,8 +232,12 @@ def test_config3_long_reasoning_whole_step(trl):
     dH = f64(out["dHidden"][torch.as_tensor(rows[sel], device=DEV)])
     ref_dH = np.stack([orc.row_dhidden(f64(batch["hidden"][int(rows[i])]), W64, ids[rows[i]], ref_g[i]) for i in sel])
     assert rel_fro(dH, ref_dH) <= TOL_GRAD
+    np.testing.assert_allclose(f64(out["g"])[rows], ref_g, rtol=2e-2, atol=1e-12)
     valid = (torch.arange(w.T, device=DEV)[None, :] < batch["lens"][:, None]).reshape(-1)
-    assert not out["dHidden"][~valid].any()
+    assert not out["dHidden"][~valid].any() and not out["g"][~valid].any()
+    col = out["dW"].double().sum(dim=0)
+    assert float(col.abs().max()) <= 1e-2 * float(out["dW"].double().abs().sum(dim=0).max())
+    assert torch.isfinite(out["dW"]).all() and torch.isfinite(out["loss"]).all()
 
 
 def _sweep_cases():
@@ -279,3 +302,34 @@ def test_config4_shape_sweep(trl, V, H, G):
     mask = torch.ones(w.N, dtype=torch.bool, device=DEV)
     mask[idx] = False
     assert not dH[mask].any()
+    del dH, dW, lse_in, g_in
+
+    # the fused schedule at the same shape (the forward's lse as the shift): log-probs, g and
+    # dHidden on the sampled rows against the oracle, and the invariants of the full outputs
+    status.zero_()
+    fo = trl.trl_pg_step_fused(batch["hidden"], batch["W"], batch["ids"], batch["lens"], old, lse, hrd["adv"], hrd["seg"],
+                               w.P, w.G, w.T, status=status)
+    torch.cuda.synchronize()
+    trl.check_status(status)
+    assert np.abs(f64(fo["logp"])[rows] - ref_logp).max() <= TOL_LOGP
+    assert abs(float(fo["loss"]) - float(loss)) <= TOL_LOSS * abs(float(loss)) + 1e-9
+    s_ratio = np.exp(ref_logp - f64(old)[rows])
+    A = ref["adv"][rows]
+    wgt = np.where(ref["seg"][rows] == 1, 0.1, 1.0)
+    active = A * s_ratio <= A * np.clip(s_ratio, 0.8, 1.2)
+    ref_g = np.where(active, -wgt * A * s_ratio / (w.P * w.G * lens[rows // w.T]), 0.0)
+    np.testing.assert_allclose(f64(fo["g"])[rows], ref_g, rtol=2e-2, atol=1e-12)
+    unit = -np.exp(z - ref_lse[:, None])
+    unit[np.arange(len(rows)), ids[rows]] += 1.0
+    ref_dH = ref_g[:, None] * (unit @ W64)
+    got = f64(fo["dHidden"][idx])
+    nz = np.linalg.norm(ref_dH, axis=1) > 0
+    if nz.any():
+        assert rel_fro(got[nz], ref_dH[nz]) <= TOL_GRAD
+    assert not got[~nz].any()
+    valid = (torch.arange(w.T, device=DEV)[None, :] < batch["lens"][:, None]).reshape(-1)
+    assert not fo["dHidden"][~valid].any() and not fo["g"][~valid].any()
+    assert not fo["g"][torch.as_tensor(ref["adv"] == 0, device=DEV)].any()
+    col = fo["dW"].double().sum(dim=0)
+    assert float(col.abs().max()) <= 1e-2 * float(fo["dW"].double().abs().sum(dim=0).max()) + 1e-30
+    assert torch.isfinite(fo["dW"]).all()

@@ -20,7 +20,8 @@ def trl():
 
 
 def run_and_compare(trl, w, batch=None, explicit_old=False, alpha=0.1, eps=0.2, adv_mode=0, fused=False,
-                    use_hint=True, clip_form=0, agg_mode=0):
+                    use_hint=True, clip_form=0, agg_mode=0, eps_hi=None):
+    eps_hi = eps if eps_hi is None else eps_hi
     dev = "cuda:0"
     batch = synth.make_batch(w, device=dev) if batch is None else batch
     oi = oracle_inputs(batch)
@@ -31,10 +32,10 @@ def run_and_compare(trl, w, batch=None, explicit_old=False, alpha=0.1, eps=0.2, 
         old_logp_o = (lp + oi["old_noise"]).astype(np.float32).astype(np.float64)
         old_logp_g = torch.tensor(old_logp_o, dtype=torch.float32, device=dev)
     ref = orc.full_step(oi["hidden"], oi["W"], oi["hidden_old"], oi["W_old"], oi["ids"], oi["lens"], oi["bnd"],
-                        oi["r_plan"], oi["r_code"], w.P, w.G, w.T, eps, eps, alpha, adv_mode, old_logp=old_logp_o,
+                        oi["r_plan"], oi["r_code"], w.P, w.G, w.T, eps, eps_hi, alpha, adv_mode, old_logp=old_logp_o,
                         clip_form=clip_form, agg_mode=agg_mode)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
-    out = trl.hrd_pg_step(batch, w.P, w.G, w.T, eps, eps, alpha, adv_mode, old_logp=old_logp_g, status=status,
+    out = trl.hrd_pg_step(batch, w.P, w.G, w.T, eps, eps_hi, alpha, adv_mode, old_logp=old_logp_g, status=status,
                           fused=fused, use_hint=use_hint, clip_form=clip_form, agg_mode=agg_mode)
     torch.cuda.synchronize()
     trl.check_status(status)
@@ -286,3 +287,146 @@ def test_minimum_workspace_gives_same_backward(trl):
     torch.cuda.synchronize()
     assert torch.equal(dH1, dH2)
     assert rel_fro(f64(dW2), f64(dW1)) < 1e-5
+
+
+# ---------------------------------------------------------------- a confident (trained) policy
+def _confident(name, scale, dtype="bf16"):
+    return synth.scaled(synth.CONFIGS[2], name=f"{name}_{scale}_{dtype}", P=2, G=4, T=300, H=320, V=1000, dtype=dtype,
+                        logit_scale=float(scale), greedy_ids=True)
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("fused", [False, True])
+@pytest.mark.parametrize("scale,med_lo,med_hi", [(8, 0.55, 0.85), (20, 0.96, 0.995), (32, 0.997, 0.9999)])
+def test_confident_policy_every_element_and_most_confident_rows(trl, dtype, fused, scale, med_lo, med_hi):
+    """Peaked softmax: the sampled token is the arg-max and carries most of the probability
+    (median p_t about 0.7, 0.98, 0.998), the regime of a trained policy.  Every output against the
+    oracle at the usual tolerances, then dHidden row by row on the most confident rows that still
+    have a gradient: there the one-hot entry g (1 - p_t) is a small difference of nearly equal
+    numbers, and the row is only right if that entry is formed without cancellation."""
+    w = _confident("confident", scale, dtype)
+    out, ref = run_and_compare(trl, w, fused=fused)
+    valid = ref["seg"] != 0
+    p_t = np.exp(ref["logp"])
+    assert med_lo <= np.median(p_t[valid]) <= med_hi
+    live = np.nonzero(valid & (ref["g"] != 0))[0]
+    # The fused step forms the entry as -sum_{v != t} E_v and is exact however small 1 - p_t is.  The
+    # separate backward recomputes p_t = exp(z_t - lse) from an lse it receives in fp32, so its entry
+    # carries an absolute error of about ulp(lse): rows with 1 - p_t below ~1e-3 are left to the
+    # Frobenius check above, where their (tiny) gradients weigh nothing.
+    floor = 1e-7 if (fused and dtype == "bf16") else 2e-3
+    cand = live[(1.0 - p_t[live]) >= floor]
+    top = cand[np.argsort(p_t[cand])[::-1][:48]]
+    assert top.size >= 16 and (1.0 - p_t[top]).min() < 2e-2
+    dH = f64(out["dHidden"])[top]
+    err = np.linalg.norm(dH - ref["dHidden"][top], axis=1) / np.linalg.norm(ref["dHidden"][top], axis=1)
+    assert err.max() <= 2e-2, (err.max(), float(p_t[top[np.argmax(err)]]))
+
+
+def test_fused_step_is_as_accurate_as_the_separate_calls_on_a_confident_policy(trl):
+    """Relative Frobenius error of dHidden and dW: the fused schedule (E stored in bf16) must stay
+    within 1.5x of the four-call schedule (dS stored in bf16), both far inside the tolerance."""
+    for scale in (8, 20, 32):
+        w = _confident("confident_cmp", scale)
+        errs = {}
+        for fused in (False, True):
+            out, ref = run_and_compare(trl, w, fused=fused)
+            errs[fused] = (rel_fro(f64(out["dHidden"]), ref["dHidden"]), rel_fro(f64(out["dW"]), ref["dW"]))
+        for k in (0, 1):
+            assert errs[True][k] <= max(1.5 * errs[False][k], 3e-3), (scale, errs)
+
+
+def test_asymmetric_clip_range(trl):
+    """eps_lo != eps_hi, old policy far enough away that both clip sides fire."""
+    w = synth.scaled(synth.CONFIGS[2], name="asym_clip", P=2, G=4, T=200, H=256, V=1536, sigma_old=0.25)
+    for fused in (False, True):
+        out, ref = run_and_compare(trl, w, fused=fused, eps=0.1, eps_hi=0.3)
+        assert ref["stats"][0] > 0.01 and ref["stats"][1] > 0.05          # both sides clip somewhere
+        assert ref["stats"][1] > 1.5 * ref["stats"][0]                    # and the narrow side clips more
+    run_and_compare(trl, w, eps=0.3, eps_hi=0.05, clip_form=1)
+    run_and_compare(trl, synth.scaled(w, name="asym_clip_f32", dtype="f32"), eps=0.3, eps_hi=0.05)
+
+
+@pytest.mark.parametrize("offset", [-60.0, -35.0, -20.0, 20.0, 45.0, 60.0])
+def test_fused_step_hint_tens_of_units_off(trl, offset):
+    """A shift c that misses the true log-partition by 20 to 60 (E then lives around e^-offset)
+    must still give the oracle's results: the header promises any hint within ~80."""
+    w = synth.scaled(synth.CONFIGS[2], name="fused_hint_far", P=2, G=4, T=200, H=256, V=1536)
+    batch = synth.make_batch(w, device="cuda:0")
+    oi = oracle_inputs(batch)
+    ref = orc.full_step(oi["hidden"], oi["W"], oi["hidden_old"], oi["W_old"], oi["ids"], oi["lens"], oi["bnd"],
+                        oi["r_plan"], oi["r_code"], w.P, w.G, w.T)
+    old_logp, old_lse = trl.trl_token_logprobs(batch["hidden_old"], batch["W_old"], batch["ids"], batch["lens"], w.T)
+    hrd = trl.trl_hrd_advantages(batch["r_plan"], batch["r_code"], batch["lens"], batch["bnd"], w.P, w.G, w.T)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda:0")
+    hint = old_lse + offset + 5.0 * (torch.rand_like(old_lse) - 0.5)
+    out = trl.trl_pg_step_fused(batch["hidden"], batch["W"], batch["ids"], batch["lens"], old_logp, hint, hrd["adv"],
+                                hrd["seg"], w.P, w.G, w.T, status=status)
+    torch.cuda.synchronize()
+    trl.check_status(status)
+    assert np.abs(f64(out["logp"]) - ref["logp"]).max() <= TOL_LOGP
+    assert abs(float(out["loss"]) - ref["loss"]) <= TOL_LOSS * abs(ref["loss"])
+    assert rel_fro(f64(out["dHidden"]), ref["dHidden"]) <= TOL_GRAD and rel_fro(f64(out["dW"]), ref["dW"]) <= TOL_GRAD
+
+
+# ---------------------------------------------------------------- long rollouts: several token tiles per rollout
+@pytest.mark.parametrize("T", [16384, 20000, 40001])
+def test_advantages_and_loss_over_several_token_tiles(trl, T):
+    """Responses up to the paper's 16,384-token limit and beyond: the advantage kernel then covers a
+    rollout with several CTAs (8192 tokens each) and the loss kernel with several partial sums
+    (16384 tokens each); T % 16 == 0, T % 4 == 0 and odd T take the three store paths."""
+    P, G = 2, 3
+    B, N = P * G, P * G * T
+    g = torch.Generator().manual_seed(T)
+    lens = torch.randint(T // 3, T + 1, (B,), generator=g, dtype=torch.int32)
+    lens[1], lens[4] = T, 8192
+    bnd = (lens.double() * torch.rand(B, generator=g, dtype=torch.float64)).to(torch.int32)
+    r_plan = torch.rand(B, generator=g) * 2.0
+    r_code = (torch.rand(B, generator=g) < 0.5).float()
+    old = -torch.rand(N, generator=g) * 6
+    logp = old + 0.15 * torch.randn(N, generator=g)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda:0")
+    dev = lambda t: t.to("cuda:0")
+    hrd = trl.trl_hrd_advantages(dev(r_plan), dev(r_code), dev(lens), dev(bnd), P, G, T, status=status)
+    loss, gg, stats = trl.trl_pg_loss_fwd(dev(logp), dev(old), hrd["adv"], hrd["seg"], dev(lens), P, G, T, status=status)
+    torch.cuda.synchronize()
+    trl.check_status(status)
+    ref = orc.hrd_advantages(f64(r_plan), f64(r_code), lens.numpy(), bnd.numpy(), P, G, T)
+    np.testing.assert_array_equal(hrd["seg"].cpu().numpy(), ref["seg"])
+    np.testing.assert_array_equal(hrd["n_plan"].cpu().numpy(), ref["n_plan"])
+    np.testing.assert_array_equal(hrd["n_code"].cpu().numpy(), ref["n_code"])
+    assert int(hrd["n_valid"].item()) == ref["n_valid"]
+    np.testing.assert_allclose(f64(hrd["adv"]), ref["adv"], rtol=1e-6, atol=1e-7)
+    rl, rg, rs = orc.pg_loss_fwd(f64(logp), f64(old), ref["adv"], ref["seg"], lens.numpy(), P, G, T)
+    assert abs(float(loss) - rl) <= TOL_LOSS * abs(rl)
+    assert rel_fro(f64(gg), rg) <= 1e-5
+    np.testing.assert_allclose(f64(stats), rs, rtol=1e-4, atol=1e-6)
+
+
+def test_fused_step_leaves_a_bad_id_row_out_of_loss_g_and_gradients(trl):
+    """A token id outside [0, V): flagged, and the row is treated as padding by everything the
+    fused call returns (same results as with that row's advantage set to zero)."""
+    w = synth.scaled(synth.CONFIGS[2], name="bad_fused", P=1, G=2, T=128, H=64, V=512)
+    batch = synth.make_batch(w, device="cuda:0")
+    batch["lens"] = torch.tensor([100, 128], dtype=torch.int32, device="cuda:0")
+    batch["bnd"] = torch.tensor([40, 60], dtype=torch.int32, device="cuda:0")
+    batch["r_plan"] = torch.tensor([1.0, 0.0], device="cuda:0")
+    batch["r_code"] = torch.tensor([0.0, 1.0], device="cuda:0")
+    old_logp, old_lse = trl.trl_token_logprobs(batch["hidden_old"], batch["W_old"], batch["ids"], batch["lens"], w.T)
+    hrd = trl.trl_hrd_advantages(batch["r_plan"], batch["r_code"], batch["lens"], batch["bnd"], w.P, w.G, w.T)
+    assert float(hrd["adv"][5]) != 0.0
+    bad = batch["ids"].clone()
+    bad[5] = 70000
+    status = torch.zeros(1, dtype=torch.int32, device="cuda:0")
+    out = trl.trl_pg_step_fused(batch["hidden"], batch["W"], bad, batch["lens"], old_logp, old_lse, hrd["adv"], hrd["seg"],
+                                w.P, w.G, w.T, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 1 << 7
+    adv0 = hrd["adv"].clone()
+    adv0[5] = 0.0
+    ref = trl.trl_pg_step_fused(batch["hidden"], batch["W"], batch["ids"], batch["lens"], old_logp, old_lse, adv0, hrd["seg"],
+                                w.P, w.G, w.T)
+    torch.cuda.synchronize()
+    assert float(out["g"][5]) == 0.0 and float(out["logp"][5]) == 0.0 and not out["dHidden"][5].any()
+    assert float(out["loss"]) == float(ref["loss"]) and torch.equal(out["dHidden"], ref["dHidden"])
+    assert torch.equal(out["g"], ref["g"]) and rel_fro(f64(out["dW"]), f64(ref["dW"])) < 1e-6

@@ -359,14 +359,64 @@ def test_backward_closed_form_at_uniform_logits():
             assert abs(dW[v, k] - ref) < 1e-14
 
 
-def test_full_step_composes():
-    p = _tiny_problem(20)
-    Wo = p["W"] + 0.05 * _rng(21).standard_normal(p["W"].shape) * p["H"] ** -0.5
-    out = orc.full_step(p["hidden"], p["W"], p["hidden"], Wo, p["ids"], p["lens"], p["bnd"],
-                        p["r_plan"], p["r_code"], p["P"], p["G"], p["T"])
-    old, _ = orc.token_logprobs(p["hidden"], Wo, p["ids"], p["lens"], p["T"])
-    np.testing.assert_array_equal(out["old_logp"], old)
-    assert np.isfinite(out["loss"]) and out["dW"].shape == p["W"].shape
+@pytest.mark.parametrize("given_old", [False, True])
+@pytest.mark.parametrize("opts", [dict(), dict(alpha=0.37, adv_mode=1), dict(clip_form=1, agg_mode=1, eps_lo=0.1, eps_hi=0.3),
+                                  dict(alpha=0.0, eps_lo=0.3, eps_hi=0.05)])
+def test_full_step_is_the_four_functions_wired_in_order(given_old, opts):
+    """Every output of full_step equals the four pinned functions composed by hand: a wrong wiring
+    (swapped policy / old-policy inputs, an option not passed on, lse of the wrong model in the
+    backward, old_logp ignored or not) changes at least one of them."""
+    p = _tiny_problem(20, P=2, G=4, T=7)
+    P, G, T = p["P"], p["G"], p["T"]
+    r = _rng(21)
+    Wo = p["W"] + 0.3 * r.standard_normal(p["W"].shape) * p["H"] ** -0.5
+    ho = p["hidden"] + 0.2 * r.standard_normal(p["hidden"].shape)
+    given = (-r.random(P * G * T) * 3.0) if given_old else None
+    out = orc.full_step(p["hidden"], p["W"], ho, Wo, p["ids"], p["lens"], p["bnd"], p["r_plan"], p["r_code"], P, G, T,
+                        old_logp=given, **opts)
+    logp, lse = orc.token_logprobs(p["hidden"], p["W"], p["ids"], p["lens"], T)
+    old = given if given_old else orc.token_logprobs(ho, Wo, p["ids"], p["lens"], T)[0]
+    hrd = orc.hrd_advantages(p["r_plan"], p["r_code"], p["lens"], p["bnd"], P, G, T, opts.get("adv_mode", 0))
+    loss, g, stats = orc.pg_loss_fwd(logp, old, hrd["adv"], hrd["seg"], p["lens"], P, G, T, opts.get("eps_lo", 0.2),
+                                     opts.get("eps_hi", 0.2), opts.get("alpha", 0.1), opts.get("clip_form", 0),
+                                     opts.get("agg_mode", 0))
+    dH, dW = orc.pg_loss_bwd(p["hidden"], p["W"], p["ids"], p["lens"], lse, g, T)
+    assert np.abs(g).max() > 0 and (not given_old or np.abs(old - orc.token_logprobs(ho, Wo, p["ids"], p["lens"], T)[0]).max() > 0.1)
+    for k, v in dict(logp=logp, lse=lse, old_logp=old, g=g, stats=stats, dHidden=dH, dW=dW, seg=hrd["seg"],
+                     adv=hrd["adv"], A_plan=hrd["A_plan"], A_code=hrd["A_code"], n_plan=hrd["n_plan"],
+                     n_code=hrd["n_code"]).items():
+        np.testing.assert_array_equal(out[k], v, err_msg=k)
+    assert out["loss"] == loss and out["n_valid"] == hrd["n_valid"]
+    # and the options do change the result (so passing them on is observable)
+    if opts:
+        base = orc.full_step(p["hidden"], p["W"], ho, Wo, p["ids"], p["lens"], p["bnd"], p["r_plan"], p["r_code"], P, G, T,
+                             old_logp=given)
+        assert base["loss"] != out["loss"]
+
+
+def test_dW_rows_is_the_row_subset_of_the_full_gradient_and_matches_loops():
+    """dW_rows against (i) the rows of pg_loss_bwd's dW (itself pinned by finite differences) with
+    arbitrary lse / g inputs, including duplicated and never-sampled vocabulary rows, and (ii) plain
+    Python loops over the definition."""
+    p = _tiny_problem(40, P=2, G=3, T=6, H=5, V=13)
+    T, V = p["T"], p["V"]
+    r = _rng(41)
+    N = p["P"] * p["G"] * T
+    lse = r.standard_normal(N) + 2.0           # not the true lse on purpose: both routines take it as given
+    g = r.standard_normal(N)
+    _, dW = orc.pg_loss_bwd(p["hidden"], p["W"], p["ids"], p["lens"], lse, g, T)
+    vsel = np.array([12, 0, 7, 7, 3])
+    got = orc.dW_rows(p["hidden"], p["W"][vsel], vsel, p["ids"], p["lens"], lse, g, T)
+    np.testing.assert_allclose(got, dW[vsel], atol=1e-13)
+    for k, v in enumerate(vsel):
+        for h in range(p["H"]):
+            acc = 0.0
+            for b in range(p["P"] * p["G"]):
+                for t in range(p["lens"][b]):
+                    n = b * T + t
+                    z = sum(p["hidden"][n, q] * p["W"][v, q] for q in range(p["H"]))
+                    acc += g[n] * ((1.0 if p["ids"][n] == v else 0.0) - math.exp(z - lse[n])) * p["hidden"][n, h]
+            assert abs(got[k, h] - acc) < 1e-12
 
 
 # ------------------------------------------------------------ documented variants of the loss

@@ -27,7 +27,9 @@ def test_static_scratch_variant_matches_workspace_variant_twice_in_a_row():
     trl.load_library()
     # two calls in a row with different shapes and data: the second one runs over whatever
     # the first left in the shared scratch array
-    for (P, G, T, seed) in ((3, 5, 9000, 1), (2, 4, 300, 2)):
+    # (the first case spans three partial-sum slots per rollout, the last one a single slot)
+    from oracle import trl_oracle as orc
+    for (P, G, T, seed) in ((2, 3, 40000, 3), (3, 5, 9000, 1), (2, 4, 300, 2)):
         logp, old, adv, seg, lens = _inputs(P, G, T, seed)
         ref_loss, ref_g, ref_stats = trl.trl_pg_loss_fwd(logp, old, adv, seg, lens, P, G, T, 0.2, 0.2, 0.1)
         loss = torch.full((1,), float("nan"), device="cuda")
@@ -41,6 +43,12 @@ def test_static_scratch_variant_matches_workspace_variant_twice_in_a_row():
         assert abs(float(loss) - float(ref_loss)) <= 1e-3 * abs(float(ref_loss)) + 1e-9
         np.testing.assert_allclose(g.cpu().numpy(), ref_g.cpu().numpy(), rtol=1e-6, atol=1e-12)
         np.testing.assert_allclose(stats.cpu().numpy(), ref_stats.cpu().numpy(), rtol=1e-6)
+        # and against the fp64 oracle, at the tolerance of the loss parity tests
+        f64 = lambda t: t.cpu().double().numpy()
+        o_loss, o_g, o_stats = orc.pg_loss_fwd(f64(logp), f64(old), f64(adv), seg.cpu().numpy(), lens.cpu().numpy(), P, G, T)
+        assert abs(float(loss) - o_loss) <= 1e-3 * abs(o_loss) + 1e-9
+        assert np.linalg.norm(f64(g) - o_g) <= 1e-5 * np.linalg.norm(o_g)
+        np.testing.assert_allclose(f64(stats), o_stats, rtol=1e-4, atol=1e-6)
 
 
 def test_static_scratch_variant_rejects_oversize():
