@@ -235,6 +235,12 @@ int trl_pg_loss_fwd_static(const float* logp, const float* old_logp, const float
  * counterpart in the paper. */
 unsigned long long trl_kernel_launches(void);
 
+/* Host string naming the tuning settings in effect, "cta_group_fwd=<n> cta_group_bwd=<n>": how many
+ * CTAs share one tensor-core instruction in the forward and in the gradient GEMMs (1, or 2 for
+ * cluster pairs).  The environment variable TRL_CTA_GROUP=1|2, read at the first call, overrides the
+ * build's default for both; results are the same either way.  No counterpart in the paper. */
+const char* trl_config_string(void);
+
 /* Host string for a status code (static storage). */
 const char* trl_status_string(int status);
 

@@ -33,6 +33,7 @@ _SIGNATURES = {
     "trl_workspace_bytes_min": (_sz, [_i, _i, _i, _i, _i, _i]),
     "trl_status_string": (ctypes.c_char_p, [_i]),
     "trl_kernel_launches": (ctypes.c_ulonglong, []),
+    "trl_config_string": (ctypes.c_char_p, []),
     "trl_token_logprobs": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _vp, _vp, _sz, _vp, _vp]),
     "trl_hrd_advantages": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "trl_pg_loss_fwd": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, PgConfig, _vp, _vp, _vp, _vp, _sz, _vp, _vp]),
@@ -100,6 +101,10 @@ def trl_workspace_bytes_min(which, B, T, H, V, dt):
 
 def trl_status_string(code):
     return load_library().trl_status_string(code).decode()
+
+
+def trl_config_string():
+    return load_library().trl_config_string().decode()
 
 
 def trl_kernel_launches():

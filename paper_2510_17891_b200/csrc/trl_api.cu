@@ -1,6 +1,8 @@
 // extern "C" entry points of libtrl: argument checks, workspace carving, kernel sequencing.
 #include <atomic>
+#include <cstdio>
 #include <cstring>
+#include <mutex>
 
 #include "trl_internal.h"
 
@@ -10,9 +12,10 @@ namespace {
 
 constexpr int kRecommendedChunkRowsBf16 = 32768;
 constexpr int kRecommendedChunkRowsF32 = 2048;
+// 128-row blocks whose tiles are rasterised together (their A rows stay in L2 while B streams)
 constexpr int kRasterBandFwd = 32;
-constexpr int kRasterBandFwdE = 16;   // forward 256x256 tiles that also store E / dS (in CTA tiles)
-constexpr int kRasterBandBwd = 4;
+constexpr int kRasterBandFwdE = 32;   // forward tiles that also store E / dS
+constexpr int kRasterBandBwd = 8;
 
 int check_device() {      // the current device must be compute capability 10.x (cached per device)
   static std::atomic<int> cached[64];      // 0: not looked up yet; otherwise status + 1
@@ -130,6 +133,15 @@ size_t trl_workspace_bytes_min(int which_call, int B, int T, int H, int V, trl_d
 
 unsigned long long trl_kernel_launches(void) { return launches_so_far(); }
 
+const char* trl_config_string(void) {
+  static char buf[64];
+  static std::once_flag once;
+  std::call_once(once, [] {
+    snprintf(buf, sizeof(buf), "cta_group_fwd=%d cta_group_bwd=%d", tc_default_cta_group(1), tc_default_cta_group(0));
+  });
+  return buf;
+}
+
 const char* trl_status_string(int status) {
   switch (status) {
     case TRL_OK: return "ok";
@@ -177,7 +189,7 @@ int trl_token_logprobs(const void* hidden, const void* W, const int32_t* ids, co
     g.A = Xp; g.a_rows = cap_rows; g.a_ld = H;
     g.B = W; g.b_rows = V; g.b_ld = H;
     g.K = H; g.N = V;
-    g.rb = rb; g.blk_off = 0; g.blk_cap = rb.cap; g.raster_band = kRasterBandFwd;
+    g.rb = rb; g.blk_off = 0; g.blk_cap = rb.cap; g.raster_band_blocks = kRasterBandFwd;
     g.ids = ids; g.partials = partials; g.tgt = tgt; g.rows_cap = cap_rows; g.status = status_dev;
     TRL_CUDA_OK(launch_tc_gemm(g, s));
     launch_merge_lse(partials, tgt, nt, cap_rows, rb, ids, len, B, T, V, logp, lse, status_dev, s);
@@ -283,19 +295,19 @@ int trl_pg_loss_bwd(const void* hidden, const void* W, const int32_t* ids, const
       a.rb = rb; a.blk_off = blk_off; a.blk_cap = CB; a.status = status_dev; a.blk_active = blk_active + blk_off;
       // dS chunk = g (onehot - softmax), from a recomputed logits tile
       TcGemm ds = a;
-      ds.epi = TC_EPI_DS; ds.raster_band = kRasterBandFwdE;
+      ds.epi = TC_EPI_DS; ds.raster_band_blocks = kRasterBandFwdE;
       ds.A = Xp; ds.a_rows = cap_rows; ds.a_ld = H; ds.B = W; ds.b_rows = V; ds.b_ld = H; ds.K = H; ds.N = V;
       ds.ids = ids; ds.lse = lse; ds.g = g; ds.dS = dS; ds.ds_ld = V;
       TRL_CUDA_OK(launch_tc_gemm(ds, s));
       // dHidden rows of the chunk = dS W   (W read as an N-contiguous operand)
       TcGemm dh = a;
-      dh.epi = TC_EPI_DH; dh.raster_band = kRasterBandBwd;
+      dh.epi = TC_EPI_DH; dh.raster_band_blocks = kRasterBandBwd;
       dh.A = dS; dh.a_rows = R; dh.a_ld = V; dh.B = W; dh.b_rows = H; dh.b_ld = H; dh.K = V; dh.N = H;
       dh.dHidden = (__nv_bfloat16*)dHidden; dh.dh_ld = H;
       TRL_CUDA_OK(launch_tc_gemm(dh, s));
       // dW += dS^T hidden   (both operands M/N-contiguous: dS [R,V] and the chunk's packed rows [.,H])
       TcGemm dw = a;
-      dw.epi = TC_EPI_DW; dw.raster_band = kRasterBandBwd;
+      dw.epi = TC_EPI_DW; dw.raster_band_blocks = kRasterBandBwd;
       dw.A = dS; dw.a_rows = V; dw.a_ld = V; dw.K = R; dw.N = H;
       dw.B = Xp + (size_t)blk_off * kRowBlock * H; dw.b_rows = H; dw.b_ld = H;
       dw.b_k = cap_rows - blk_off * kRowBlock < R ? cap_rows - blk_off * kRowBlock : R;
@@ -392,7 +404,7 @@ int trl_pg_step_fused(const void* hidden, const void* W, const int32_t* ids, con
     float* tgt_all = cv.take<float>(cap_rows);
     float2* partials = cv.take<float2>((size_t)nt * cap_rows);
     TcGemm f = base;
-    f.epi = TC_EPI_LSE; f.raster_band = kRasterBandFwd;
+    f.epi = TC_EPI_LSE; f.raster_band_blocks = kRasterBandFwd;
     f.A = Xp; f.a_rows = cap_rows; f.a_ld = H; f.B = W; f.b_rows = V; f.b_ld = H; f.K = H; f.N = V;
     f.blk_off = 0; f.blk_cap = rb.cap; f.ids = ids; f.partials = partials; f.tgt = tgt_all; f.rows_cap = cap_rows;
     TRL_CUDA_OK(launch_tc_gemm(f, s));
@@ -406,7 +418,7 @@ int trl_pg_step_fused(const void* hidden, const void* W, const int32_t* ids, con
     a.blk_off = blk_off; a.blk_cap = CB;
     // forward tile -> E = exp(z - c), row sums, sampled token's logit
     TcGemm e = a;
-    e.epi = TC_EPI_E; e.raster_band = kRasterBandFwdE;
+    e.epi = TC_EPI_E; e.raster_band_blocks = kRasterBandFwdE;
     e.A = Xp; e.a_rows = cap_rows; e.a_ld = H; e.B = W; e.b_rows = V; e.b_ld = H; e.K = H; e.N = V;
     e.ids = ids; e.lse = hint; e.dS = E; e.ds_ld = V; e.psum = psum; e.tgt = tgt; e.rows_cap = R;
     TRL_CUDA_OK(launch_tc_gemm(e, s));
@@ -416,13 +428,13 @@ int trl_pg_step_fused(const void* hidden, const void* W, const int32_t* ids, con
     launch_pack_rows_bf16(Xp, Xs, H, R, rb, blk_off * kRowBlock, 1, neg_alpha, s);
     // dHidden rows = neg_alpha * (E' W)
     TcGemm dh = a;
-    dh.epi = TC_EPI_DH; dh.raster_band = kRasterBandBwd;
+    dh.epi = TC_EPI_DH; dh.raster_band_blocks = kRasterBandBwd;
     dh.A = E; dh.a_rows = R; dh.a_ld = V; dh.B = W; dh.b_rows = H; dh.b_ld = H; dh.K = V; dh.N = H;
     dh.dHidden = (__nv_bfloat16*)dHidden; dh.dh_ld = H; dh.row_scale = neg_alpha; dh.blk_active = blk_active;
     TRL_CUDA_OK(launch_tc_gemm(dh, s));
     // dW += E'^T (neg_alpha * hidden)
     TcGemm dw = a;
-    dw.epi = TC_EPI_DW; dw.raster_band = kRasterBandBwd;
+    dw.epi = TC_EPI_DW; dw.raster_band_blocks = kRasterBandBwd;
     dw.A = E; dw.a_rows = V; dw.a_ld = V; dw.B = Xs; dw.b_rows = H; dw.b_ld = H; dw.K = R; dw.N = H;
     dw.m_blocks = cdiv(V, kRowBlock); dw.dW = dW; dw.dw_ld = H; dw.V = V; dw.blk_active = blk_active;
     TRL_CUDA_OK(launch_tc_gemm(dw, s));

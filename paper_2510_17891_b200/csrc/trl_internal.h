@@ -102,7 +102,8 @@ struct TcGemm {
   int N;                                     // GEMM N extent = b_rows that are meaningful
   int m_blocks;                              // TC_EPI_DW: fixed number of 128-row blocks of A; others: from row blocks
   RowPack rb; int blk_off, blk_cap;        // chunk of row blocks
-  int raster_band;
+  int raster_band_blocks;                    // 128-row blocks rasterised together (0: default)
+  int cta_group;                             // CTAs per MMA: 1, 2 (cluster pairs), 0: the build's default
   // epilogue arguments
   const int32_t* ids; const float* lse; const float* g;
   float2* partials; float* tgt; int rows_cap;          // LSE
@@ -117,5 +118,6 @@ struct TcGemm {
 // returns cudaSuccess or the error of tensor-map creation / launch
 cudaError_t launch_tc_gemm(const TcGemm& p, cudaStream_t s);
 int tc_num_sms();
+int tc_default_cta_group(int fwd);   // CTAs per MMA in effect for the forward (1) / gradient (0) GEMMs
 
 }  // namespace trl

@@ -28,6 +28,7 @@
 #include <cuda.h>
 
 #include <atomic>
+#include <cstdlib>
 
 #include "trl_internal.h"
 
@@ -35,10 +36,21 @@ namespace trl {
 
 namespace {
 
-constexpr int BM = 128, BN = 256, BK = 64, UMMA_K = 16, STAGES = 4;
-constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
+// CTAs per MMA for the forward GEMMs (LSE, dS, E) and the gradient GEMMs (dHidden, dW): 1, or 2
+// for cluster pairs (tcgen05 cta_group::2)
+#ifndef TRL_CTA_GROUP_FWD
+#define TRL_CTA_GROUP_FWD 1
+#endif
+#ifndef TRL_CTA_GROUP_BWD
+#define TRL_CTA_GROUP_BWD 1
+#endif
+
+constexpr int BM = 128, BN = 256, BK = 64, UMMA_K = 16;
+constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2;
+constexpr int RING_BYTES = 4 * (A_BYTES + B_BYTES);   // 192 KB of operand stages, cut into 3 to 6 stages
+constexpr int MAX_STAGES = 6;
 constexpr int OUT_STAGE_BYTES = 4 * 2 * 4096;   // 4 epilogue warps x 2 buffers x (32 rows x 128 B)
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + OUT_STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int SMEM_BYTES = RING_BYTES + OUT_STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr float LOG2E = 1.4426950408889634f, LN2 = 0.6931471805599453f;
 constexpr long long WAIT_CYCLES = 4000000000LL;   // ~2-3 s at B200 clocks
@@ -100,6 +112,51 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm,
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
       ::"r"(dst), "l"(tm), "r"(bar), "r"(x), "r"(y)
+      : "memory");
+}
+// ---- CTA pairs (cta_group::2).  The two CTAs of a cluster share one MMA: each holds its own 128
+// rows of A and half of the B tile in its own shared memory, the even CTA ("leader") issues the
+// instruction, and each CTA's tensor memory receives its own 128 accumulator rows.  Every copy is a
+// plain TMA load into the issuing CTA's own shared memory; only its completion is signalled on the
+// leader's barrier.
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// shared::cluster address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+}
+// load into this CTA's shared memory; the bytes are counted on `cluster_bar`, a barrier of the pair's leader
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t cluster_bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(tm), "r"(cluster_bar), "r"(x), "r"(y)
+      : "memory");
+}
+// arrives on the barrier at this shared-memory offset in both CTAs of the pair once all earlier MMAs are done
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
+  asm volatile(
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+      ::"r"(bar), "h"((uint16_t)3)
+      : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16_pair(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
+                                                 uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -387,48 +444,58 @@ __device__ __forceinline__ void epilogue_tile(const TcArgs& p, uint32_t tmem_acc
 }
 
 // ---------------------------------------------------------------- the kernel
-// MT = 128-row M blocks per CTA tile.  The scoring GEMM (LSE) uses MT = 1 and alternates
-// between two TMEM accumulators so the epilogue overlaps the next mainloop.  All other GEMMs
-// use MT = 2: one B tile in shared memory feeds both accumulators, which cuts the shared-memory
-// fill traffic per FLOP by a third, and the epilogue runs exposed.  For the gradient GEMMs
-// (K = V or K = rows of a chunk) it is 0.4-2 % of the mainloop; for the forward GEMMs that
-// store dS / E (K = H) two epilogue warp groups drain the two accumulators at the same time.
-template <int EPI> struct TileCfg {
-  static constexpr int MT = (EPI == TC_EPI_LSE) ? 1 : 2;
+// CG = CTAs that share one MMA (tcgen05 cta_group): 1, or 2 for a cluster pair.
+// MT = accumulators (128-row M blocks) per CTA and tile.
+//   CG = 1: the scoring GEMM (LSE) uses MT = 1 and alternates between two TMEM accumulators so
+//     the epilogue overlaps the next mainloop; all other GEMMs use MT = 2, one B tile in shared
+//     memory feeding both accumulators, with the epilogue exposed (two epilogue warp groups drain
+//     the two accumulators of the forward GEMMs that store dS / E).
+//   CG = 2: a pair works on 256 x 256 (forward GEMMs, MT = 1, two alternating accumulators per
+//     CTA) or 512 x 256 (gradient GEMMs, MT = 2) and each CTA stages only its own A rows and half
+//     of the B tile: a third to a half less shared-memory traffic per FLOP than CG = 1.
+// M block of accumulator j of tile ms in the CTA of rank r: (ms * MT + j) * CG + r.
+template <int EPI, int CG> struct TileCfg {
+  static constexpr bool FWD = (EPI == TC_EPI_LSE || EPI == TC_EPI_E || EPI == TC_EPI_DS);
+  static constexpr int MT = (CG == 2) ? (FWD ? 1 : 2) : ((EPI == TC_EPI_LSE) ? 1 : 2);
   // epilogue warp groups (4 warps each) working in parallel, one accumulator each
-  static constexpr int EG = (EPI == TC_EPI_E || EPI == TC_EPI_DS) ? 2 : 1;
+  static constexpr int EG = (CG == 1 && (EPI == TC_EPI_E || EPI == TC_EPI_DS)) ? 2 : 1;
   static constexpr int THREADS = 64 + 128 * EG;
   static constexpr int NACC = 2 / MT;                       // accumulator sets in the 512 TMEM columns
-  static constexpr int STG_BYTES = MT * A_BYTES + B_BYTES;  // 48 KB or 64 KB
-  static constexpr int NSTAGE = (STAGES * STAGE_BYTES) / STG_BYTES;   // 4 or 3
+  static constexpr int BN_CTA = BN / CG;                    // rows of the B tile this CTA stages
+  static constexpr int STG_BYTES = MT * A_BYTES + B_BYTES / CG;   // 48 / 64 KB (CG 1), 32 / 48 KB (CG 2)
+  static constexpr int NSTAGE = RING_BYTES / STG_BYTES;           // 4 / 3, 6 / 4
+  static_assert(NSTAGE <= MAX_STAGES && NSTAGE >= 2, "stage count");
 };
 
-template <int EPI>
-__global__ void __launch_bounds__(TileCfg<EPI>::THREADS, 1)
+template <int EPI, int CG>
+__global__ void __launch_bounds__(TileCfg<EPI, CG>::THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmOut, const TcArgs p) {
-  using Cfg = TileCfg<EPI>;
+  using Cfg = TileCfg<EPI, CG>;
   constexpr int MT = Cfg::MT, NACC = Cfg::NACC, NSTAGE = Cfg::NSTAGE, STG = Cfg::STG_BYTES, EG = Cfg::EG;
+  constexpr int BN_CTA = Cfg::BN_CTA;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t out_base = smem_base + STAGES * STAGE_BYTES;          // 1024-aligned
+  const uint32_t out_base = smem_base + RING_BYTES;                    // 1024-aligned
   const uint32_t bar_base = out_base + OUT_STAGE_BYTES;
-  // barrier layout (8 B each): full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2]; then tmem slot, abort flag
+  // barrier layout (8 B each): full[MAX_STAGES], empty[MAX_STAGES], tmem_full[2], tmem_empty[2]; then tmem slot, abort flag
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
-  auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
-  auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
-  auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (MAX_STAGES + s); };
+  auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * MAX_STAGES + a); };
+  auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * MAX_STAGES + 2 + a); };
   uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen_base + STAGES * STAGE_BYTES + OUT_STAGE_BYTES + 8 * (2 * STAGES + 4));
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen_base + STAGES * STAGE_BYTES + OUT_STAGE_BYTES + 8 * (2 * STAGES + 4) + 8);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen_base + RING_BYTES + OUT_STAGE_BYTES + 8 * (2 * MAX_STAGES + 4));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen_base + RING_BYTES + OUT_STAGE_BYTES + 8 * (2 * MAX_STAGES + 4) + 8);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int rank = (CG == 2) ? (int)cluster_ctarank() : 0;        // 0 = the CTA that issues the MMAs
+  const int worker = (int)blockIdx.x / CG, n_workers = (int)gridDim.x / CG;   // CTAs (CG 1) or pairs (CG 2)
 
-  // ---- problem extents (identical in every thread)
+  // ---- problem extents (identical in every thread, and in both CTAs of a pair)
   int live = p.blk_cap;
   if (p.nblk) live = max(0, min(p.nblk[0] - p.blk_off, p.blk_cap));
   const int MB = (EPI == TC_EPI_DW) ? p.m_blocks_fixed : live;    // 128-row blocks
-  const int MS = (MB + MT - 1) / MT;                               // CTA tiles along M
+  const int MS = (MB + MT * CG - 1) / (MT * CG);                   // tiles along M
   const int K = (EPI == TC_EPI_DW) ? live * BM : p.K;
   const int NT = (p.N + BN - 1) / BN;
   const int nkb = (K + BK - 1) / BK;
@@ -438,74 +505,92 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     for (int i = 0; i < live; ++i) n_act += p.blk_active[i] != 0;
     if (n_act == 0) total = 0;
   }
-  if (total == 0 || (int)blockIdx.x >= total) return;
-  // Which M sub-blocks of a CTA tile take part (identical decision in every role): present, and for
-  // dS / dHidden not marked inactive.  Which k-blocks take part: for dW, those of active row blocks.
+  if (total == 0 || worker >= total) return;        // the same decision in both CTAs of a pair
+  // Is M block mb worked on at all: present, and for dS / dHidden not marked inactive.
+  auto blk_on = [&](int mb) {
+    return mb < MB && (!((EPI == TC_EPI_DH || EPI == TC_EPI_DS) && p.blk_active) || p.blk_active[mb] != 0);
+  };
+  // Which accumulators of a tile take part (identical decision in every role and in both CTAs): an
+  // accumulator spans the M blocks of all CG CTAs and runs if any of them is worked on.  Which
+  // k-blocks take part: for dW, those of active row blocks.
   auto tile_mask = [&](int ms) {
-    const int nm = min(MT, MB - ms * MT);
     int m = 0;
-    for (int j = 0; j < nm; ++j)
-      if (!((EPI == TC_EPI_DH || EPI == TC_EPI_DS) && p.blk_active) || p.blk_active[ms * MT + j] != 0) m |= 1 << j;
+    for (int j = 0; j < MT; ++j)
+      for (int r = 0; r < CG; ++r)
+        if (blk_on((ms * MT + j) * CG + r)) m |= 1 << j;
     return m;
   };
   auto kb_on = [&](int kb) { return !(EPI == TC_EPI_DW && p.blk_active) || p.blk_active[kb >> 1] != 0; };
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 128 * EG); }
+    for (int s = 0; s < MAX_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 128 * EG * CG); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 1) {
+  if (warp == 1) {           // with CG = 2 the same warp of both CTAs allocates, at the same shared-memory offset
     __syncwarp();
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void*)tmem_slot)),
-                 "r"(TMEM_COLS)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if constexpr (CG == 2) {
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void*)tmem_slot)),
+                   "r"(TMEM_COLS)
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void*)tmem_slot)),
+                   "r"(TMEM_COLS)
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
   }
   tc_fence_before();
   __syncthreads();
+  if constexpr (CG == 2) cluster_sync_all();     // the partner's barriers exist before anything signals them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   auto a_row_of = [&](int mb) {
     // forward GEMMs read the packed hidden rows of the block; the gradient GEMMs read chunk scratch
-    return (EPI == TC_EPI_LSE || EPI == TC_EPI_DS || EPI == TC_EPI_E) ? (p.blk_off + mb) * BM : mb * BM;
+    return Cfg::FWD ? (p.blk_off + mb) * BM : mb * BM;
   };
 
   if (warp == 0) {
-    // ------------------------------------------------------------ TMA producer
+    // ------------------------------------------------------------ TMA producer (one per CTA)
     if (lane == 0) {
       int stage = 0; uint32_t phase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x) {
+      for (int tile = worker; tile < total && ok; tile += n_workers) {
         int ms, nt;
         tile_coords(tile, MS, NT, p.raster_band, ms, nt);
-        const int mask = tile_mask(ms);                        // M blocks of this tile that take part
+        const int mask = tile_mask(ms);                        // accumulators of this tile that take part
         if (mask == 0) continue;
-        const int b_row = nt * BN;
+        const int b_row = nt * BN + rank * BN_CTA;
         for (int kb = 0; kb < nkb; ++kb) {
           if (!kb_on(kb)) continue;
           if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status))) break;
-          mbar_expect_tx(full_bar(stage), (uint32_t)(__popc(mask) * A_BYTES + B_BYTES));
+          // bytes of this stage over all CTAs of the pair, expected on the leader's barrier
+          if (rank == 0) mbar_expect_tx(full_bar(stage), (uint32_t)(CG * (__popc(mask) * A_BYTES + B_BYTES / CG)));
+          const uint32_t fb = (CG == 2) ? map_to_cta(full_bar(stage), 0) : full_bar(stage);
+          auto load = [&](uint32_t dst, const CUtensorMap* tm, int x, int y) {
+            if constexpr (CG == 2) tma_load_2d_pair(dst, tm, x, y, fb); else tma_load_2d(dst, tm, x, y, fb);
+          };
           const uint32_t sa = smem_base + stage * STG;
 #pragma unroll
           for (int j = 0; j < MT; ++j) {
             if (mask & (1 << j)) {
-              const int a_row = a_row_of(ms * MT + j);
+              const int a_row = a_row_of((ms * MT + j) * CG + rank);
               if constexpr (a_is_mn(EPI)) {       // two 64(M) x 64(K) boxes
-                tma_load_2d(sa + j * A_BYTES, &tmA, a_row, kb * BK, full_bar(stage));
-                tma_load_2d(sa + j * A_BYTES + 8192, &tmA, a_row + 64, kb * BK, full_bar(stage));
+                load(sa + j * A_BYTES, &tmA, a_row, kb * BK);
+                load(sa + j * A_BYTES + 8192, &tmA, a_row + 64, kb * BK);
               } else {
-                tma_load_2d(sa + j * A_BYTES, &tmA, kb * BK, a_row, full_bar(stage));
+                load(sa + j * A_BYTES, &tmA, kb * BK, a_row);
               }
             }
           }
           const uint32_t sb = sa + MT * A_BYTES;
-          if constexpr (b_is_mn(EPI)) {       // four 64(N) x 64(K) boxes
+          if constexpr (b_is_mn(EPI)) {       // 64(N) x 64(K) boxes
 #pragma unroll
-            for (int j = 0; j < BN / 64; ++j) tma_load_2d(sb + j * 8192, &tmB, b_row + 64 * j, kb * BK, full_bar(stage));
+            for (int j = 0; j < BN_CTA / 64; ++j) load(sb + j * 8192, &tmB, b_row + 64 * j, kb * BK);
           } else {
-            tma_load_2d(sb, &tmB, kb * BK, b_row, full_bar(stage));
+            load(sb, &tmB, kb * BK, b_row);
           }
           if (++stage == NSTAGE) { stage = 0; phase ^= 1u; }
         }
@@ -516,13 +601,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
     __syncwarp();
   } else if (warp == 1) {
-    // ------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      constexpr uint32_t idesc = make_idesc_bf16(BM, BN, a_is_mn(EPI), b_is_mn(EPI));
+    // ------------------------------------------------------------ MMA issuer (the leader's, for a pair)
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = make_idesc_bf16(BM * CG, BN, a_is_mn(EPI), b_is_mn(EPI));
       int stage = 0; uint32_t phase = 0;
       int acc = 0; uint32_t acc_phase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x) {
+      auto commit = [&](uint32_t bar) { if constexpr (CG == 2) tc_commit_pair(bar); else tc_commit(bar); };
+      for (int tile = worker; tile < total && ok; tile += n_workers) {
         int ms, nt;
         tile_coords(tile, MS, NT, p.raster_band, ms, nt);
         const int mask = tile_mask(ms);
@@ -546,16 +632,19 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             if (mask & (1 << j)) {
               const uint64_t da = a_is_mn(EPI) ? make_mnmajor_sw128_desc(sa + j * A_BYTES) : make_kmajor_sw128_desc(sa + j * A_BYTES);
 #pragma unroll
-              for (int k = 0; k < BK / UMMA_K; ++k)
-                tc_mma_bf16(d_tmem + (uint32_t)(j * BN), da + ka * k, db + kbs * k, idesc, (uint32_t)(!(first_kb && k == 0)));
+              for (int k = 0; k < BK / UMMA_K; ++k) {
+                const uint32_t accum = (uint32_t)(!(first_kb && k == 0));
+                if constexpr (CG == 2) tc_mma_bf16_pair(d_tmem + (uint32_t)(j * BN), da + ka * k, db + kbs * k, idesc, accum);
+                else tc_mma_bf16(d_tmem + (uint32_t)(j * BN), da + ka * k, db + kbs * k, idesc, accum);
+              }
             }
           }
           first_kb = false;
-          tc_commit(empty_bar(stage));
+          commit(empty_bar(stage));
           if (++stage == NSTAGE) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
-        tc_commit(tfull_bar(acc));
+        commit(tfull_bar(acc));
         if (++acc == NACC) { acc = 0; acc_phase ^= 1u; }
       }
     }
@@ -566,7 +655,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int grp = (warp - 2) / 4;      // group g drains the accumulators j with j % EG == g
     WarpOut wo{out_base + (uint32_t)(warp - 2) * (8192u / EG), &tmOut, lane, 0, 2 / EG};
     int acc = 0; uint32_t acc_phase = 0;
-    for (int tile = blockIdx.x; tile < total; tile += gridDim.x) {
+    for (int tile = worker; tile < total; tile += n_workers) {
       int ms, nt;
       tile_coords(tile, MS, NT, p.raster_band, ms, nt);
       const int mask = tile_mask(ms);
@@ -576,10 +665,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       if (!ok) break;
       tc_fence_after();
 #pragma unroll
-      for (int j = 0; j < MT; ++j)
-        if ((mask & (1 << j)) && (j % EG) == grp) epilogue_tile<EPI>(p, tmem_base + (uint32_t)((acc * MT + j) * BN), quad, lane, ms * MT + j, nt, wo);
+      for (int j = 0; j < MT; ++j) {
+        const int mb = (ms * MT + j) * CG + rank;       // this CTA's M block of accumulator j
+        if ((mask & (1 << j)) && (j % EG) == grp && blk_on(mb))
+          epilogue_tile<EPI>(p, tmem_base + (uint32_t)((acc * MT + j) * BN), quad, lane, mb, nt, wo);
+      }
       tc_fence_before();
-      mbar_arrive(tempty_bar(acc));
+      if constexpr (CG == 2) mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));    // the leader's MMA issuer waits on it
+      else mbar_arrive(tempty_bar(acc));
       if (++acc == NACC) { acc = 0; acc_phase ^= 1u; }
     }
     wo.drain();      // staged stores must have left shared memory before the CTA exits
@@ -587,10 +680,16 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
   tc_fence_before();
   __syncthreads();
+  // a pair leaves together: the leader's MMAs read the partner's shared memory and the partner's
+  // epilogue signals the leader's barriers
+  if constexpr (CG == 2) cluster_sync_all();
   if (warp == 1) {
     __syncwarp();
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    if constexpr (CG == 2)
+      asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    else
+      asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
   }
 }
 
@@ -642,21 +741,70 @@ bool make_out_tmap(CUtensorMap* tm, void* base, long inner, long outer, long ld,
   return r == CUDA_SUCCESS;
 }
 
-template <int EPI>
-cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmOut, const TcArgs& a, int grid,
+template <int EPI, int CG>
+cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmOut, const TcArgs& a, int workers,
                        cudaStream_t s) {
   static std::atomic<bool> attr_set[64];   // the attribute is per device; setting it twice is harmless
   int dev = 0;
   cudaGetDevice(&dev);
   if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
   if (!attr_set[dev].load(std::memory_order_acquire)) {
-    cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel<EPI, CG>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (e != cudaSuccess) return e;
     attr_set[dev].store(true, std::memory_order_release);
   }
-  tc_gemm_kernel<EPI><<<grid, TileCfg<EPI>::THREADS, SMEM_BYTES, s>>>(tmA, tmB, tmOut, a);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(workers * CG));
+  cfg.blockDim = dim3((unsigned)TileCfg<EPI, CG>::THREADS);
+  cfg.dynamicSmemBytes = SMEM_BYTES;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = CG; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = (CG > 1) ? 1 : 0;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, tc_gemm_kernel<EPI, CG>, tmA, tmB, tmOut, a);
   note_launch();
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
+}
+
+template <int CG>
+cudaError_t launch_cg(const TcGemm& g, cudaStream_t s) {
+  CUtensorMap tmA, tmB;
+  if (!make_tmap(&tmA, g.A, g.a_rows, g.K, g.a_ld, BM, a_is_mn(g.epi))) return cudaErrorInvalidValue;
+  if (!make_tmap(&tmB, g.B, g.b_rows, g.b_k > 0 ? g.b_k : g.K, g.b_ld, BN / CG, b_is_mn(g.epi))) return cudaErrorInvalidValue;
+  CUtensorMap tmOut = tmA;      // unused by the LSE and DH epilogues
+  if (g.epi == TC_EPI_DS || g.epi == TC_EPI_E) {
+    if (!make_out_tmap(&tmOut, g.dS, g.N, (long)g.blk_cap * BM, g.ds_ld, false)) return cudaErrorInvalidValue;
+  } else if (g.epi == TC_EPI_DW) {
+    if (!make_out_tmap(&tmOut, g.dW, g.N, g.V, g.dw_ld, true)) return cudaErrorInvalidValue;
+  }
+  TcArgs a;
+  a.N = g.N; a.K = g.K; a.m_blocks_fixed = g.m_blocks; a.blk_off = g.blk_off; a.blk_cap = g.blk_cap;
+  a.rows_cap = g.rows_cap; a.V = g.V;
+  a.nblk = g.rb.nblk; a.n_rows = g.rb.n_rows; a.rowmap = g.rb.rowmap;
+  a.ids = g.ids; a.lse = g.lse; a.g = g.g; a.partials = g.partials; a.tgt = g.tgt;
+  a.dS = g.dS; a.ds_ld = g.ds_ld;
+  a.dHidden = g.dHidden; a.dh_ld = g.dh_ld; a.dW = g.dW; a.dw_ld = g.dw_ld; a.status = g.status;
+  a.psum = g.psum; a.row_scale = g.row_scale; a.blk_active = g.blk_active;
+  const bool fwd = (g.epi == TC_EPI_LSE || g.epi == TC_EPI_E || g.epi == TC_EPI_DS);
+  const int mt = (CG == 2) ? (fwd ? 1 : 2) : (g.epi == TC_EPI_LSE ? 1 : 2);     // as TileCfg
+  // rows of M tiles rasterised together, so that their A rows stay in L2 while B streams: the
+  // caller gives it in 128-row blocks
+  a.raster_band = (g.raster_band_blocks > 0 ? g.raster_band_blocks : 32) / (mt * CG);
+  if (a.raster_band < 1) a.raster_band = 1;
+  const int NT = cdiv(g.N, BN);
+  const long max_tiles = (long)cdiv(g.epi == TC_EPI_DW ? g.m_blocks : g.blk_cap, mt * CG) * NT;
+  const int slots = tc_num_sms() / CG;
+  const int workers = (int)(max_tiles < (long)slots ? (max_tiles > 0 ? max_tiles : 1) : slots);
+  switch (g.epi) {
+    case TC_EPI_LSE: return launch_one<TC_EPI_LSE, CG>(tmA, tmB, tmOut, a, workers, s);
+    case TC_EPI_DS: return launch_one<TC_EPI_DS, CG>(tmA, tmB, tmOut, a, workers, s);
+    case TC_EPI_DH: return launch_one<TC_EPI_DH, CG>(tmA, tmB, tmOut, a, workers, s);
+    case TC_EPI_DW: return launch_one<TC_EPI_DW, CG>(tmA, tmB, tmOut, a, workers, s);
+    case TC_EPI_E: return launch_one<TC_EPI_E, CG>(tmA, tmB, tmOut, a, workers, s);
+  }
+  return cudaErrorInvalidValue;
 }
 
 }  // namespace
@@ -674,36 +822,22 @@ int tc_num_sms() {
   return v > 0 ? v : 1;
 }
 
+// CTAs per MMA when the caller leaves it open: the build's default, or TRL_CTA_GROUP=1|2 from the
+// environment (read once).  Pairs do a few % more work per clock (less shared-memory traffic), but
+// on a power-capped B200 they draw more power per FLOP and end up slower, so 1 is the default.
+static int default_cta_group(bool fwd) {
+  static const int env = [] {
+    const char* e = getenv("TRL_CTA_GROUP");
+    return (e && (e[0] == '1' || e[0] == '2') && e[1] == 0) ? e[0] - '0' : 0;
+  }();
+  return env ? env : (fwd ? TRL_CTA_GROUP_FWD : TRL_CTA_GROUP_BWD);
+}
+
+int tc_default_cta_group(int fwd) { return default_cta_group(fwd != 0); }
+
 cudaError_t launch_tc_gemm(const TcGemm& g, cudaStream_t s) {
-  CUtensorMap tmA, tmB;
-  if (!make_tmap(&tmA, g.A, g.a_rows, g.K, g.a_ld, BM, a_is_mn(g.epi))) return cudaErrorInvalidValue;
-  if (!make_tmap(&tmB, g.B, g.b_rows, g.b_k > 0 ? g.b_k : g.K, g.b_ld, BN, b_is_mn(g.epi))) return cudaErrorInvalidValue;
-  CUtensorMap tmOut = tmA;      // unused by the LSE and DH epilogues
-  if (g.epi == TC_EPI_DS || g.epi == TC_EPI_E) {
-    if (!make_out_tmap(&tmOut, g.dS, g.N, (long)g.blk_cap * BM, g.ds_ld, false)) return cudaErrorInvalidValue;
-  } else if (g.epi == TC_EPI_DW) {
-    if (!make_out_tmap(&tmOut, g.dW, g.N, g.V, g.dw_ld, true)) return cudaErrorInvalidValue;
-  }
-  TcArgs a;
-  a.N = g.N; a.K = g.K; a.m_blocks_fixed = g.m_blocks; a.blk_off = g.blk_off; a.blk_cap = g.blk_cap;
-  a.raster_band = g.raster_band > 0 ? g.raster_band : 16; a.rows_cap = g.rows_cap; a.V = g.V;
-  a.nblk = g.rb.nblk; a.n_rows = g.rb.n_rows; a.rowmap = g.rb.rowmap;
-  a.ids = g.ids; a.lse = g.lse; a.g = g.g; a.partials = g.partials; a.tgt = g.tgt;
-  a.dS = g.dS; a.ds_ld = g.ds_ld;
-  a.dHidden = g.dHidden; a.dh_ld = g.dh_ld; a.dW = g.dW; a.dw_ld = g.dw_ld; a.status = g.status;
-  a.psum = g.psum; a.row_scale = g.row_scale; a.blk_active = g.blk_active;
-  const int NT = cdiv(g.N, BN);
-  const int mt = (g.epi == TC_EPI_LSE) ? 1 : 2;
-  const long max_tiles = (long)cdiv(g.epi == TC_EPI_DW ? g.m_blocks : g.blk_cap, mt) * NT;
-  const int grid = (int)(max_tiles < (long)tc_num_sms() ? (max_tiles > 0 ? max_tiles : 1) : tc_num_sms());
-  switch (g.epi) {
-    case TC_EPI_LSE: return launch_one<TC_EPI_LSE>(tmA, tmB, tmOut, a, grid, s);
-    case TC_EPI_DS: return launch_one<TC_EPI_DS>(tmA, tmB, tmOut, a, grid, s);
-    case TC_EPI_DH: return launch_one<TC_EPI_DH>(tmA, tmB, tmOut, a, grid, s);
-    case TC_EPI_DW: return launch_one<TC_EPI_DW>(tmA, tmB, tmOut, a, grid, s);
-    case TC_EPI_E: return launch_one<TC_EPI_E>(tmA, tmB, tmOut, a, grid, s);
-  }
-  return cudaErrorInvalidValue;
+  const int cg = g.cta_group > 0 ? g.cta_group : default_cta_group(!(g.epi == TC_EPI_DH || g.epi == TC_EPI_DW));
+  return cg == 2 ? launch_cg<2>(g, s) : launch_cg<1>(g, s);
 }
 
 }  // namespace trl
