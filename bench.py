@@ -220,7 +220,17 @@ class StepRunner:
                          stats=torch.empty(4, **f32), dHidden=torch.empty_like(batch["hidden"]),
                          dW=torch.empty(V, H, **f32), ws_fwd=ws(trl.TRL_CALL_TOKEN_LOGPROBS),
                          ws_loss=ws(trl.TRL_CALL_PG_LOSS_FWD),
-                         ws_bwd=ws(trl.TRL_CALL_PG_LOSS_BWD if path == "four_call" else trl.TRL_CALL_PG_STEP_FUSED))
+                         ws_bwd=ws(trl.TRL_CALL_PG_LOSS_BWD if path == "four_call" else trl.TRL_CALL_PG_STEP_FUSED)
+                         if not (dp_allreduce and path == "fused") else None)
+        # data-parallel training: dW is finished band by band and every band is all-reduced on a side
+        # stream as soon as it is final (with one rank: the banded schedule alone)
+        self.reducer = None
+        if dp_allreduce and path == "fused":
+            from paper_2510_17891_b200 import dp
+            self.rows_bound = int(batch["lens"].sum().item())
+            self.bufs["ws_bwd"] = torch.empty(trl.trl_pg_step_fused_banded_workspace_bytes(B, T, H, V, self.rows_bound),
+                                              dtype=torch.uint8, device=dev)
+            self.reducer = dp.BandedGradReducer(self.bufs["dW"], trl.trl_dw_band_plan(V, H, 16), w.P)
         self.fused_out = {k: self.bufs[k] for k in ("logp", "lse", "g", "loss", "stats", "dHidden", "dW")}
         self.status = torch.zeros(1, dtype=torch.int32, device=dev)
         self.stream = torch.cuda.current_stream()
@@ -250,7 +260,15 @@ class StepRunner:
                                      bufs.get("hrd"), status, stream)
         bufs["hrd"] = hrd
         mark()
-        if self.path == "fused":
+        if self.reducer is not None:
+            self.reducer.finish()          # the previous step's dW is reduced before this step overwrites it
+            trl.trl_pg_step_fused_banded(batch["hidden"], batch["W"], batch["ids"], batch["lens"], bufs["old_logp"],
+                                         bufs["old_lse"], hrd["adv"], hrd["seg"], P, G, T, self.reducer.band_begin,
+                                         self.reducer.events, self.rows_bound, 0.2, 0.2, 0.1, self.fused_out, bufs["ws_bwd"],
+                                         status, stream)
+            self.reducer.start(bufs["loss"])
+            self.reducer.finish()
+        elif self.path == "fused":
             trl.trl_pg_step_fused(batch["hidden"], batch["W"], batch["ids"], batch["lens"], bufs["old_logp"], bufs["old_lse"],
                                   hrd["adv"], hrd["seg"], P, G, T, 0.2, 0.2, 0.1, self.fused_out, bufs["ws_bwd"], status, stream)
         else:
@@ -260,7 +278,7 @@ class StepRunner:
             trl.trl_pg_loss_bwd(batch["hidden"], batch["W"], batch["ids"], batch["lens"], bufs["lse"], bufs["g"], T,
                                 bufs["dHidden"], bufs["dW"], bufs["ws_bwd"], status, stream)
         mark()
-        if self.dp_allreduce and self.dist is not None:
+        if self.dp_allreduce and self.reducer is None and self.dist is not None:      # four_call: all-reduce after the step
             from paper_2510_17891_b200 import dp
             dp.allreduce_step_outputs(bufs["dW"], bufs["loss"], P)
 
@@ -327,7 +345,8 @@ def main():
     ap.add_argument("--reductions", action="store_true",
                     help="time the two memory-bound calls (HRD advantages, surrogate loss) alone at 2^26 tokens")
     ap.add_argument("--dp-allreduce", action="store_true",
-                    help="N > 1 only: also all-reduce dW and the loss across ranks every step (data-parallel training)")
+                    help="data-parallel training: run the banded schedule (dW final band by band) and, with N > 1, "
+                         "all-reduce every band of dW and the loss across ranks on a side stream as it becomes final")
     ap.add_argument("--path", default="fused", choices=["fused", "four_call"],
                     help="fused: old-policy scoring, advantages, trl_pg_step_fused; four_call: the separate calls")
     args = ap.parse_args()
@@ -482,7 +501,7 @@ def main():
                     dtype=w.dtype, data="synthetic",
                     config=dict(workload=w.name, P=P, G=G, T=T, H=H, V=V, valid_tokens_per_rank=n_valid,
                                 padded_rows_per_rank=B * T, l2="inputs larger than L2 (W alone is 1.2 GB); no flush",
-                                parallelism=(f"data-parallel x{world}, dW + loss all-reduced every step" if args.dp_allreduce and world > 1
+                                parallelism=(f"data-parallel x{world}, dW all-reduced band by band behind the dW GEMM, loss all-reduced" if args.dp_allreduce
                                              else f"replicas x{world} (independent batches)")),
                     pct_of_bf16_peak_6NHV=dict(nominal=100 * step_alg / 2250.0,
                                                measured_sustained=100 * step_alg / peaks["bf16_sustained"],

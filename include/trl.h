@@ -60,7 +60,8 @@ typedef enum {
   TRL_ERR_CUDA = 6,       /* a CUDA runtime / driver call failed   */
   TRL_ERR_BAD_INDEX = 7,  /* device-detected: id, len or bnd out of range */
   TRL_ERR_TIMEOUT = 8,    /* device-detected: a bounded pipeline wait expired */
-  TRL_ERR_BAD_HINT = 9    /* device-detected: lse_hint so far off that exp(z - hint) left the fp32 range */
+  TRL_ERR_BAD_HINT = 9,   /* device-detected: lse_hint so far off that exp(z - hint) left the fp32 range */
+  TRL_ERR_ROWS_BOUND = 10 /* device-detected: more valid rows than the caller's rows_bound (trl_pg_step_fused_banded) */
 } trl_status;
 
 /* Storage type of hidden / W / dHidden.  TRL_BF16 runs on the tcgen05 tensor cores with
@@ -205,6 +206,42 @@ int trl_pg_step_fused(const void* hidden, const void* W, const int32_t* ids, con
                       float* logp, float* lse, float* loss, float* g, float* stats,
                       void* dHidden, float* dW,
                       void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream);
+
+/*
+ * trl_pg_step_fused for data-parallel training: same inputs, outputs and results (bit for bit),
+ * but dW becomes final band by band, so that its reduction across ranks can overlap the rest of
+ * the dW GEMM.  The paper trains on 8 GPUs (training-details appendix) without describing how; the
+ * path shards by prompt group, and the LM-head gradient is the one tensor the ranks must sum.
+ *
+ * E = exp(z - c) is kept for all rows instead of one chunk (workspace:
+ * trl_pg_step_fused_banded_workspace_bytes, about rows_bound * V * 2 bytes more), the forward and
+ * the dHidden GEMM run chunk by chunk as before, and then the dW GEMM runs once per band of
+ * vocabulary rows [band_begin[j], band_begin[j+1]) over all chunks.  After the last launch of
+ * band j the event band_events[j] is recorded on `stream`: rows band_begin[j] .. band_begin[j+1]
+ * of dW are final from that point of the stream on.  The caller makes a second stream wait for
+ * the event and starts the band's all-reduce there (NCCL or its own kernel); nothing in this
+ * library communicates.
+ *
+ * n_bands, band_begin [n_bands + 1] (host): band_begin[0] = 0, band_begin[n_bands] = V, increasing,
+ *   every band_begin[j] a multiple of 256 (trl_dw_band_plan makes such a split).
+ * band_events [n_bands] (host array of cudaEvent_t, or NULL; single entries may be NULL).
+ * rows_bound: an upper bound on sum_b len[b] known on the host, or 0 for B*T.  It sizes the
+ *   workspace; if the batch has more valid rows, TRL_ERR_ROWS_BOUND is set in *status_dev and the
+ *   excess rows are dropped.
+ * TRL_BF16 only.
+ */
+int trl_pg_step_fused_banded(const void* hidden, const void* W, const int32_t* ids, const int32_t* len,
+                             const float* old_logp, const float* lse_hint, const float* adv, const uint8_t* seg,
+                             int P, int G, int T, int H, int V, trl_dtype dt, trl_pg_config cfg,
+                             float* logp, float* lse, float* loss, float* g, float* stats,
+                             void* dHidden, float* dW,
+                             int n_bands, const int32_t* band_begin, void* const* band_events, int rows_bound,
+                             void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream);
+size_t trl_pg_step_fused_banded_workspace_bytes(int B, int T, int H, int V, int rows_bound);
+/* Splits the V rows of dW into at most n_bands_wanted bands of whole 256-row tiles, sized so that
+ * each band's launch fills whole waves of CTAs.  Writes band_begin [returned count + 1] (host; give
+ * it n_bands_wanted + 1 entries) and returns the number of bands (0 on bad arguments). */
+int trl_dw_band_plan(int V, int H, int n_bands_wanted, int32_t* band_begin);
 
 /*
  * Same computation and outputs as trl_pg_loss_fwd, for callers that cannot allocate device

@@ -10,5 +10,6 @@ from .binding import (  # noqa: F401
     TrlError, PgConfig, lib_path, load_library, exported_symbols,
     trl_workspace_bytes, trl_workspace_bytes_min, trl_status_string, trl_kernel_launches, trl_config_string,
     trl_token_logprobs, trl_hrd_advantages, trl_pg_loss_fwd, trl_pg_loss_fwd_static, trl_pg_loss_bwd, trl_pg_step_fused,
+    trl_pg_step_fused_banded, trl_pg_step_fused_banded_workspace_bytes, trl_dw_band_plan,
     check_status, hrd_pg_step,
 )

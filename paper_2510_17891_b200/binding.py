@@ -7,7 +7,7 @@ import torch
 TRL_F32, TRL_BF16 = 0, 1
 TRL_CALL_TOKEN_LOGPROBS, TRL_CALL_PG_LOSS_FWD, TRL_CALL_PG_LOSS_BWD, TRL_CALL_PG_STEP_FUSED = 0, 1, 2, 3
 _STATUS_BITS = {7: "index out of range (token id / len / bnd)", 8: "pipeline wait timed out",
-                9: "lse_hint out of range"}
+                9: "lse_hint out of range", 10: "more valid rows than rows_bound"}
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
 _lib = None
@@ -39,6 +39,9 @@ _SIGNATURES = {
     "trl_pg_loss_fwd": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, PgConfig, _vp, _vp, _vp, _vp, _sz, _vp, _vp]),
     "trl_pg_loss_fwd_static": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, PgConfig, _vp, _vp, _vp, _vp, _vp]),
     "trl_pg_step_fused": (_i, [_vp] * 8 + [_i] * 6 + [PgConfig] + [_vp] * 7 + [_vp, _sz, _vp, _vp]),
+    "trl_pg_step_fused_banded": (_i, [_vp] * 8 + [_i] * 6 + [PgConfig] + [_vp] * 7 + [_i, _vp, _vp, _i] + [_vp, _sz, _vp, _vp]),
+    "trl_pg_step_fused_banded_workspace_bytes": (_sz, [_i, _i, _i, _i, _i]),
+    "trl_dw_band_plan": (_i, [_i, _i, _i, _vp]),
     "trl_pg_loss_bwd": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _vp, _vp, _sz, _vp, _vp]),
 }
 
@@ -243,6 +246,57 @@ def trl_pg_step_fused(hidden, W, ids, lens, old_logp, lse_hint, adv, seg, P, G, 
                                           _ptr(o["stats"]), _ptr(o["dHidden"]), _ptr(o["dW"]), _ptr(workspace),
                                           workspace.numel(), _ptr(status), _stream(stream))
     _check(rc, "trl_pg_step_fused")
+    return o
+
+
+def trl_dw_band_plan(V, H, n_bands_wanted):
+    """Band boundaries (a list of n + 1 vocabulary rows) for trl_pg_step_fused_banded."""
+    buf = (ctypes.c_int32 * (n_bands_wanted + 1))()
+    n = load_library().trl_dw_band_plan(V, H, n_bands_wanted, buf)
+    if n <= 0:
+        raise TrlError("trl_dw_band_plan: invalid arguments")
+    return [int(buf[i]) for i in range(n + 1)]
+
+
+def trl_pg_step_fused_banded_workspace_bytes(B, T, H, V, rows_bound=0):
+    return load_library().trl_pg_step_fused_banded_workspace_bytes(B, T, H, V, rows_bound)
+
+
+def trl_pg_step_fused_banded(hidden, W, ids, lens, old_logp, lse_hint, adv, seg, P, G, T, band_begin, band_events=None,
+                             rows_bound=0, eps_lo=0.2, eps_hi=0.2, alpha=0.1, out=None, workspace=None, status=None,
+                             stream=None, clip_form=0, agg_mode=0):
+    """trl_pg_step_fused with dW finished band by band (see include/trl.h).  `band_begin` is a list
+    of n + 1 rows from trl_dw_band_plan; `band_events` a list of n recorded-at-least-once
+    torch.cuda.Event objects (or None): event j is recorded on the stream when band j of dW is final."""
+    _dev(hidden, W, ids, lens, old_logp, lse_hint, adv, seg, workspace, status)
+    B = lens.numel()
+    V, H = W.shape
+    dt = _dt(hidden)
+    dev = hidden.device
+    o = {} if out is None else out
+    f32 = dict(dtype=torch.float32, device=dev)
+    for k, shape in (("logp", B * T), ("lse", B * T), ("g", B * T), ("loss", 1), ("stats", 4)):
+        if o.get(k) is None:
+            o[k] = torch.empty(shape, **f32)
+    if o.get("dHidden") is None:
+        o["dHidden"] = torch.empty_like(hidden)
+    if o.get("dW") is None:
+        o["dW"] = torch.empty(V, H, **f32)
+    if workspace is None:
+        workspace = _workspace(trl_pg_step_fused_banded_workspace_bytes(B, T, H, V, rows_bound), dev)
+    n = len(band_begin) - 1
+    bb = (ctypes.c_int32 * (n + 1))(*band_begin)
+    ev = None
+    if band_events is not None:
+        ev = (ctypes.c_void_p * n)(*[None if e is None else e.cuda_event for e in band_events])
+    rc = load_library().trl_pg_step_fused_banded(_ptr(hidden), _ptr(W), _ptr(ids), _ptr(lens), _ptr(old_logp), _ptr(lse_hint),
+                                                 _ptr(adv), _ptr(seg), P, G, T, H, V, dt,
+                                                 PgConfig(eps_lo, eps_hi, alpha, clip_form, agg_mode),
+                                                 _ptr(o["logp"]), _ptr(o["lse"]), _ptr(o["loss"]), _ptr(o["g"]),
+                                                 _ptr(o["stats"]), _ptr(o["dHidden"]), _ptr(o["dW"]),
+                                                 n, bb, ev, rows_bound, _ptr(workspace), workspace.numel(), _ptr(status),
+                                                 _stream(stream))
+    _check(rc, "trl_pg_step_fused_banded")
     return o
 
 

@@ -76,6 +76,22 @@ size_t fused_per_rows_bf16(int H, int V, int R) {
          2 * align_up((size_t)R * 4, 256) + align_up((size_t)(R / kRowBlock) * 4, 256);
 }
 
+// banded schedule: E, the scaled hidden rows, the row factors and the activity flags are kept for all
+// RB rows (RB = the caller's bound on the number of valid rows, rounded up to 128); row sums and
+// target logits are per chunk of Rc rows
+int banded_rows(int B, int T, int rows_bound) {
+  const int cap = rows_cap_of(B, T);
+  if (rows_bound <= 0 || rows_bound > B * T) return cap;
+  return cdiv(rows_bound, kRowBlock) * kRowBlock;
+}
+size_t fused_banded_bytes(int B, int T, int H, int V, int rows_bound, bool with_fwd_extra) {
+  const size_t RB = banded_rows(B, T, rows_bound);
+  const size_t Rc = RB < (size_t)kRecommendedChunkRowsBf16 ? RB : (size_t)kRecommendedChunkRowsBf16;
+  return fused_fixed_bf16(B, T, H, V) + align_up(RB * H * 2, 256) + align_up(RB * V * 2, 256) +
+         align_up((size_t)cdiv(V, 256) * Rc * 4, 256) + align_up(Rc * 4, 256) + align_up(RB * 4, 256) +
+         align_up((RB / kRowBlock) * 4, 256) + (with_fwd_extra ? fwd_extra_bf16(B, T, V) : 0);
+}
+
 // largest multiple of 128 rows (<= cap) whose scratch fits into `avail` bytes
 template <class F>
 int fit_rows(size_t avail, int cap, F bytes_of) {
@@ -154,6 +170,7 @@ const char* trl_status_string(int status) {
     case TRL_ERR_BAD_INDEX: return "index out of range (device)";
     case TRL_ERR_TIMEOUT: return "pipeline wait timed out (device)";
     case TRL_ERR_BAD_HINT: return "lse_hint out of range (device)";
+    case TRL_ERR_ROWS_BOUND: return "more valid rows than rows_bound (device)";
   }
   return "unknown status";
 }
@@ -337,11 +354,24 @@ int trl_pg_loss_bwd(const void* hidden, const void* W, const int32_t* ids, const
 }
 
 
-int trl_pg_step_fused(const void* hidden, const void* W, const int32_t* ids, const int32_t* len,
-                      const float* old_logp, const float* lse_hint, const float* adv, const uint8_t* seg,
-                      int P, int G, int T, int H, int V, trl_dtype dt, trl_pg_config cfg,
-                      float* logp, float* lse, float* loss, float* g, float* stats, void* dHidden, float* dW,
-                      void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream) {
+}  // extern "C"
+
+namespace {
+
+struct DwBands {            // dW finished band by band (host arrays)
+  int n; const int32_t* begin; void* const* events; int rows_bound;
+};
+
+int fused_banded(const void* hidden, const void* W, const int32_t* ids, const int32_t* len, const float* old_logp,
+                 const float* lse_hint, const float* adv, const uint8_t* seg, int P, int G, int T, int H, int V,
+                 trl_pg_config cfg, float* logp, float* lse, float* loss, float* g, float* stats, void* dHidden, float* dW,
+                 void* workspace, size_t workspace_bytes, int32_t* status_dev, cudaStream_t s, const DwBands& bands);
+
+int fused_impl(const void* hidden, const void* W, const int32_t* ids, const int32_t* len,
+               const float* old_logp, const float* lse_hint, const float* adv, const uint8_t* seg,
+               int P, int G, int T, int H, int V, trl_dtype dt, trl_pg_config cfg,
+               float* logp, float* lse, float* loss, float* g, float* stats, void* dHidden, float* dW,
+               void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream, const DwBands* bands) {
   if (!hidden || !W || !ids || !len || !old_logp || !adv || !seg || !logp || !lse || !loss || !g || !dHidden || !dW ||
       !workspace)
     return TRL_ERR_INVALID_ARG;
@@ -357,6 +387,16 @@ int trl_pg_step_fused(const void* hidden, const void* W, const int32_t* ids, con
       !al16(seg) || !al16(logp) || !al16(lse) || !al16(g) || !al4(loss) || (lse_hint && !al16(lse_hint)) || (stats && !al4(stats)) ||
       (status_dev && !al4(status_dev)))
     return TRL_ERR_INVALID_ARG;
+  if (bands) {
+    if (dt != TRL_BF16) return TRL_ERR_DTYPE;
+    if (bands->n < 1 || !bands->begin || bands->begin[0] != 0 || bands->begin[bands->n] != V) return TRL_ERR_INVALID_ARG;
+    for (int j = 0; j < bands->n; ++j)      // bands are whole 256-row tiles of dW, in order
+      if (bands->begin[j + 1] <= bands->begin[j] || (bands->begin[j] % 256) != 0) return TRL_ERR_INVALID_ARG;
+    if (workspace_bytes < fused_banded_bytes(B, T, H, V, bands->rows_bound, lse_hint == nullptr)) return TRL_ERR_WORKSPACE_TOO_SMALL;
+    if (int e = check_device()) return e;
+    return fused_banded(hidden, W, ids, len, old_logp, lse_hint, adv, seg, P, G, T, H, V, cfg, logp, lse, loss, g, stats,
+                        dHidden, dW, workspace, workspace_bytes, status_dev, (cudaStream_t)stream, *bands);
+  }
   if (workspace_bytes < trl_workspace_bytes_min(TRL_CALL_PG_STEP_FUSED, B, T, H, V, dt)) return TRL_ERR_WORKSPACE_TOO_SMALL;
   if (int e = check_device()) return e;
 
@@ -444,6 +484,156 @@ int trl_pg_step_fused(const void* hidden, const void* W, const int32_t* ids, con
   launch_pg_loss(logp, old_logp, adv, seg, len, P, G, T, cfg, loss, g, stats, loss_partials, ids, V, s);
   TRL_CUDA_OK(cudaGetLastError());
   return TRL_OK;
+}
+
+// The same step with E kept for all rows, so that the dW GEMM can run vocabulary band by vocabulary
+// band over all row chunks: a band of dW is final as soon as its launches are done, and an event
+// recorded there lets the caller start reducing it across ranks while later bands are computed.
+// Every 256-row tile of dW receives the same per-chunk contributions in the same order as in the
+// chunk-by-chunk schedule above, so the results are bit-identical to it.
+int fused_banded(const void* hidden, const void* W, const int32_t* ids, const int32_t* len, const float* old_logp,
+                 const float* lse_hint, const float* adv, const uint8_t* seg, int P, int G, int T, int H, int V,
+                 trl_pg_config cfg, float* logp, float* lse, float* loss, float* g, float* stats, void* dHidden, float* dW,
+                 void* workspace, size_t workspace_bytes, int32_t* status_dev, cudaStream_t s, const DwBands& bands) {
+  (void)workspace_bytes;
+  const int B = P * G;
+  const int cap_rows = rows_cap_of(B, T);
+  const size_t N = (size_t)B * T;
+  const int nt = cdiv(V, 256);
+  const int RB = banded_rows(B, T, bands.rows_bound);
+  const int Rc = RB < kRecommendedChunkRowsBf16 ? RB : kRecommendedChunkRowsBf16;
+
+  Carver cv(workspace);
+  RowPack rb = carve_row_pack(cv.take<char>(row_pack_bytes(B, T)), B, T);
+  __nv_bfloat16* Xp = cv.take<__nv_bfloat16>((size_t)cap_rows * H);
+  int* unused_flags = cv.take<int>(rb.cap);            // keeps the fixed part laid out as fused_fixed_bf16 counts it
+  (void)unused_flags;
+  float* loss_partials = cv.take<float>((size_t)B * pg_loss_tiles(T) * 4);
+  __nv_bfloat16* Xs = cv.take<__nv_bfloat16>((size_t)RB * H);
+  __nv_bfloat16* E = cv.take<__nv_bfloat16>((size_t)RB * V);
+  float* psum = cv.take<float>((size_t)nt * Rc);
+  float* tgt = cv.take<float>(Rc);
+  float* neg_alpha = cv.take<float>(RB);
+  int* blk_active = cv.take<int>(RB / kRowBlock);
+
+  launch_build_row_pack(len, B, T, rb, status_dev, s);
+  launch_clamp_rows(rb, RB, status_dev, s);            // more valid rows than the caller's bound: flagged, the excess is dropped
+  TRL_CUDA_OK(cudaMemsetAsync(dW, 0, (size_t)V * H * sizeof(float), s));
+  TRL_CUDA_OK(cudaMemsetAsync(dHidden, 0, N * H * 2, s));
+  launch_zero_padded_f32(logp, lse, len, B, T, s);
+  launch_pack_rows_bf16((const __nv_bfloat16*)hidden, Xp, H, cap_rows, rb, 0, 0, nullptr, s);
+
+  TcGemm base;
+  memset(&base, 0, sizeof(base));
+  base.rb = rb; base.status = status_dev;
+
+  const float* hint = lse_hint;
+  if (!hint) {
+    float* tgt_all = cv.take<float>(cap_rows);
+    float2* partials = cv.take<float2>((size_t)nt * cap_rows);
+    TcGemm f = base;
+    f.epi = TC_EPI_LSE; f.raster_band_blocks = kRasterBandFwd;
+    f.A = Xp; f.a_rows = cap_rows; f.a_ld = H; f.B = W; f.b_rows = V; f.b_ld = H; f.K = H; f.N = V;
+    f.blk_off = 0; f.blk_cap = rb.cap; f.ids = ids; f.partials = partials; f.tgt = tgt_all; f.rows_cap = cap_rows;
+    TRL_CUDA_OK(launch_tc_gemm(f, s));
+    launch_merge_lse(partials, tgt_all, nt, cap_rows, rb, ids, len, B, T, V, logp, lse, status_dev, s);
+    hint = lse;
+  }
+
+  const int CB = Rc / kRowBlock, NB = RB / kRowBlock;
+  for (int blk_off = 0; blk_off < NB; blk_off += CB) {
+    const int cb = NB - blk_off < CB ? NB - blk_off : CB;          // blocks of this chunk
+    __nv_bfloat16* Ec = E + (size_t)blk_off * kRowBlock * V;
+    TcGemm a = base;
+    a.blk_off = blk_off; a.blk_cap = cb;
+    TcGemm e = a;
+    e.epi = TC_EPI_E; e.raster_band_blocks = kRasterBandFwdE;
+    e.A = Xp; e.a_rows = cap_rows; e.a_ld = H; e.B = W; e.b_rows = V; e.b_ld = H; e.K = H; e.N = V;
+    e.ids = ids; e.lse = hint; e.dS = Ec; e.ds_ld = V; e.psum = psum; e.tgt = tgt; e.rows_cap = Rc;
+    TRL_CUDA_OK(launch_tc_gemm(e, s));
+    FusedMergeArgs m{psum, tgt, nt, Rc, rb, blk_off, ids, len, hint, old_logp, adv, seg, P, G, T, V, cfg,
+                     logp, lse, g, neg_alpha + (size_t)blk_off * kRowBlock, blk_active + blk_off, Ec, status_dev};
+    m.R_live = cb * kRowBlock;
+    launch_fused_merge(m, s);
+    launch_pack_rows_bf16(Xp, Xs + (size_t)blk_off * kRowBlock * H, H, cb * kRowBlock, rb, blk_off * kRowBlock, 1,
+                          neg_alpha + (size_t)blk_off * kRowBlock, s);
+    TcGemm dh = a;
+    dh.epi = TC_EPI_DH; dh.raster_band_blocks = kRasterBandBwd;
+    dh.A = Ec; dh.a_rows = cb * kRowBlock; dh.a_ld = V; dh.B = W; dh.b_rows = H; dh.b_ld = H; dh.K = V; dh.N = H;
+    dh.dHidden = (__nv_bfloat16*)dHidden; dh.dh_ld = H; dh.row_scale = neg_alpha + (size_t)blk_off * kRowBlock;
+    dh.blk_active = blk_active + blk_off;
+    TRL_CUDA_OK(launch_tc_gemm(dh, s));
+  }
+  for (int j = 0; j < bands.n; ++j) {
+    const int v0 = bands.begin[j], vn = bands.begin[j + 1] - v0;
+    for (int blk_off = 0; blk_off < NB; blk_off += CB) {
+      const int cb = NB - blk_off < CB ? NB - blk_off : CB;
+      TcGemm dw = base;
+      dw.blk_off = blk_off; dw.blk_cap = cb;
+      dw.epi = TC_EPI_DW; dw.raster_band_blocks = kRasterBandBwd;
+      dw.A = E + (size_t)blk_off * kRowBlock * V + v0; dw.a_rows = vn; dw.a_ld = V;
+      dw.B = Xs + (size_t)blk_off * kRowBlock * H; dw.b_rows = H; dw.b_ld = H; dw.K = cb * kRowBlock; dw.N = H;
+      dw.m_blocks = cdiv(vn, kRowBlock); dw.dW = dW + (size_t)v0 * H; dw.dw_ld = H; dw.V = vn;
+      dw.blk_active = blk_active + blk_off;
+      TRL_CUDA_OK(launch_tc_gemm(dw, s));
+    }
+    if (bands.events && bands.events[j]) TRL_CUDA_OK(cudaEventRecord((cudaEvent_t)bands.events[j], s));
+  }
+  launch_pg_loss(logp, old_logp, adv, seg, len, P, G, T, cfg, loss, g, stats, loss_partials, ids, V, s);
+  TRL_CUDA_OK(cudaGetLastError());
+  return TRL_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int trl_pg_step_fused(const void* hidden, const void* W, const int32_t* ids, const int32_t* len,
+                      const float* old_logp, const float* lse_hint, const float* adv, const uint8_t* seg,
+                      int P, int G, int T, int H, int V, trl_dtype dt, trl_pg_config cfg,
+                      float* logp, float* lse, float* loss, float* g, float* stats, void* dHidden, float* dW,
+                      void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream) {
+  return fused_impl(hidden, W, ids, len, old_logp, lse_hint, adv, seg, P, G, T, H, V, dt, cfg, logp, lse, loss, g, stats,
+                    dHidden, dW, workspace, workspace_bytes, status_dev, stream, nullptr);
+}
+
+int trl_pg_step_fused_banded(const void* hidden, const void* W, const int32_t* ids, const int32_t* len,
+                             const float* old_logp, const float* lse_hint, const float* adv, const uint8_t* seg,
+                             int P, int G, int T, int H, int V, trl_dtype dt, trl_pg_config cfg,
+                             float* logp, float* lse, float* loss, float* g, float* stats, void* dHidden, float* dW,
+                             int n_bands, const int32_t* band_begin, void* const* band_events, int rows_bound,
+                             void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream) {
+  DwBands b{n_bands, band_begin, band_events, rows_bound};
+  return fused_impl(hidden, W, ids, len, old_logp, lse_hint, adv, seg, P, G, T, H, V, dt, cfg, logp, lse, loss, g, stats,
+                    dHidden, dW, workspace, workspace_bytes, status_dev, stream, &b);
+}
+
+size_t trl_pg_step_fused_banded_workspace_bytes(int B, int T, int H, int V, int rows_bound) {
+  if (!shapes_ok(B, T, H, V)) return 0;
+  return fused_banded_bytes(B, T, H, V, rows_bound, true);
+}
+
+int trl_dw_band_plan(int V, int H, int n_bands_wanted, int32_t* band_begin) {
+  if (V <= 0 || H <= 0 || n_bands_wanted < 1 || !band_begin) return 0;
+  // Whole 256-row tiles of dW per band, as equal as possible.  A band's launch has (tiles of the
+  // band) x (tiles along H) CTA tiles; the tile count per band is rounded up to the smallest count
+  // that fills whole waves of a B200's 148 CTAs, so that no band ends in a nearly empty wave.
+  const int m_tiles = cdiv(V, 256), n_tiles = cdiv(H, 256);
+  int a = 148, b = n_tiles;
+  while (b) { const int t = a % b; a = b; b = t; }        // a = gcd(148, n_tiles)
+  const int q = 148 / a;
+  int per = cdiv(m_tiles, n_bands_wanted);
+  if (per > q) per = ((per + q / 2) / q) * q;             // nearest multiple of q
+  int n;
+  for (;;) {
+    n = cdiv(m_tiles, per);
+    if (n > 1 && (m_tiles - (n - 1) * per) * 4 < per) --n;  // a short last band joins the one before it
+    if (n <= n_bands_wanted) break;
+    per += (per >= q) ? q : 1;
+  }
+  for (int j = 0; j < n; ++j) band_begin[j] = j * per * 256;
+  band_begin[n] = V;
+  return n;
 }
 
 }  // extern "C"

@@ -37,6 +37,8 @@ void launch_hrd_advantages(const float* r_plan, const float* r_code, const int32
                            int P, int G, int T, int adv_mode, float* A_plan, float* A_code, uint8_t* seg,
                            float* adv, int32_t* n_plan, int32_t* n_code, int64_t* n_valid, int32_t* status,
                            cudaStream_t s);
+// n_rows > max_rows (a multiple of 128): flag TRL_ERR_ROWS_BOUND and drop the excess rows
+void launch_clamp_rows(RowPack rb, int max_rows, int32_t* status, cudaStream_t s);
 int  pg_loss_tiles(int T);
 // ids may be null; when given, tokens whose id is outside [0, V) are left out like padding
 void launch_pg_loss(const float* logp, const float* old_logp, const float* adv, const uint8_t* seg,
@@ -61,6 +63,7 @@ struct FusedMergeArgs {
   int* blk_active;                  // [R/128] 1 if any row of the block has a non-zero factor
   __nv_bfloat16* E;
   int32_t* status;
+  int R_live;                       // rows of the chunk that exist (0: R); R stays the stride of psum
 };
 void launch_fused_merge(const FusedMergeArgs& a, cudaStream_t s);
 // blk_active[i] = 1 if any of the 128 packed rows of row block i has g != 0 (i < nblk)

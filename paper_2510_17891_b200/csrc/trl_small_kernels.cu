@@ -84,6 +84,18 @@ void launch_build_row_pack(const int32_t* len, int B, int T, RowPack rb, int32_t
   note_launch();
 }
 
+__global__ void clamp_rows_kernel(RowPack rb, int max_rows, int32_t* status) {
+  if (rb.n_rows[0] > max_rows) {
+    flag_status(status, TRL_ERR_ROWS_BOUND);
+    rb.n_rows[0] = max_rows;
+    rb.nblk[0] = max_rows / kRowBlock;
+  }
+}
+void launch_clamp_rows(RowPack rb, int max_rows, int32_t* status, cudaStream_t s) {
+  clamp_rows_kernel<<<1, 1, 0, s>>>(rb, max_rows, status);
+  note_launch();
+}
+
 // ------------------------------------------------------------------------------------
 // HRD advantages.  grid = (token tiles, B).  Each CTA re-derives its group's means with a
 // warp-shuffle reduction over the G rewards of the prompt (fp64), then streams out the
@@ -454,9 +466,10 @@ __global__ void __launch_bounds__(128) fused_merge_kernel(FusedMergeArgs a) {
   // one CTA = one 128-row block of the chunk
   const int r = blockIdx.x * 128 + threadIdx.x;
   const int q = a.blk_off * kRowBlock + r;
-  if (blockIdx.x * 128 >= a.R || a.blk_off + (int)blockIdx.x >= a.rb.nblk[0]) return;   // whole block not live
+  const int R_live = a.R_live > 0 ? a.R_live : a.R;
+  if (blockIdx.x * 128 >= R_live || a.blk_off + (int)blockIdx.x >= a.rb.nblk[0]) return;   // whole block not live
   float gn = 0.f;
-  if (r < a.R && q < a.rb.n_rows[0]) {
+  if (r < R_live && q < a.rb.n_rows[0]) {
     const size_t n = (size_t)a.rb.rowmap[q];
     const int b = (int)(n / a.T);
     float s_excl = 0.f;
@@ -480,7 +493,7 @@ __global__ void __launch_bounds__(128) fused_merge_kernel(FusedMergeArgs a) {
     if (gn != 0.f) a.E[(size_t)r * a.V + id] = __float2bfloat16_rn(-s_excl);
     gn = -gn * expf(c - lse);
   }
-  if (r < a.R) a.neg_alpha[r] = gn;
+  if (r < R_live) a.neg_alpha[r] = gn;
   const int any = __syncthreads_or(gn != 0.f);
   if (threadIdx.x == 0) a.blk_active[blockIdx.x] = any;
 }
@@ -500,7 +513,7 @@ void launch_flag_active_blocks(const float* g, RowPack rb, int* blk_active, cuda
 }
 
 void launch_fused_merge(const FusedMergeArgs& a, cudaStream_t s) {
-  fused_merge_kernel<<<cdiv(a.R, 128), 128, 0, s>>>(a);
+  fused_merge_kernel<<<cdiv(a.R_live > 0 ? a.R_live : a.R, 128), 128, 0, s>>>(a);
   note_launch();
 }
 

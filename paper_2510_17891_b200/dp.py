@@ -5,9 +5,11 @@ of the LM head, so scoring, advantages, loss and backward have no exchange step.
 data-parallel trainer exchanges afterwards is the LM-head gradient (and the scalar loss):
 `allreduce_step_outputs` does that with the process group's all-reduce (NCCL over NVLink on
 GPUs, gloo on CPU), in buckets so the first buckets can be reduced while later ones are
-still being enqueued.  The benchmark keeps it off by default (ranks are independent
-replicas there); its bookkeeping (time = max over ranks, tokens = sum) is in
-`aggregate_throughput`."""
+still being enqueued.  `BandedGradReducer` goes one step further together with
+`trl_pg_step_fused_banded`: the dW GEMM finishes dW band by band and records an event per band,
+and each band's all-reduce is started on a side stream behind that event while later bands are
+still being computed.  The benchmark keeps both off by default (ranks are independent replicas
+there); its bookkeeping (time = max over ranks, tokens = sum) is in `aggregate_throughput`."""
 import torch
 import torch.distributed as dist
 
@@ -52,3 +54,65 @@ def allreduce_step_outputs(dW: torch.Tensor, loss: torch.Tensor, n_prompts_local
     for wk in works:
         wk.wait()
     return int(round(tot.item()))
+
+
+class BandedGradReducer:
+    """Sums dW (and the loss) over the ranks band by band, each band as soon as it is final.
+
+    Use with trl_pg_step_fused_banded: pass `band_begin` and `events` to it; when it has returned
+    (everything is enqueued, nothing has run yet necessarily) call `start(loss)`: for every band j, in
+    band order on every rank, the side stream waits for event j, scales rows
+    band_begin[j]..band_begin[j+1] of dW by this rank's share of the prompts and starts their
+    all-reduce.  `finish()` makes the current stream wait for all of them; call it before dW is
+    read and before the next step overwrites it.  Each rank computed its loss and gradient as a mean
+    over its own P_r prompts, so the global mean over sum_r P_r prompts is
+    sum_r (P_r / P_total) * (rank r's result).
+
+    On CPU tensors (gloo) there are no streams or events: the bands are reduced in the same order
+    with the same weights, which is what the two-rank CPU test checks.  Without a process group
+    (or with one rank) nothing is communicated and dW is left untouched.
+    """
+
+    def __init__(self, dW: torch.Tensor, band_begin, n_prompts_local: int, group=None):
+        self.dW, self.band_begin, self.group = dW, list(band_begin), group
+        self.active = dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1
+        self.cuda = dW.is_cuda
+        self.n_prompts_total = n_prompts_local
+        self.weight = 1.0
+        if self.active:                       # one-off host round trip; the prompt split is fixed for a run
+            tot = torch.tensor([float(n_prompts_local)], dtype=torch.float64, device=dW.device)
+            dist.all_reduce(tot, op=dist.ReduceOp.SUM, group=group)
+            self.n_prompts_total = int(round(tot.item()))
+            self.weight = n_prompts_local / float(self.n_prompts_total)
+        n = len(self.band_begin) - 1
+        self.events, self.side = None, None
+        if self.cuda:
+            self.events = [torch.cuda.Event() for _ in range(n)]
+            for e in self.events:             # an event has a handle to pass on once it has been recorded
+                e.record()
+            self.side = torch.cuda.Stream(device=dW.device, priority=-1)
+        self.works = []
+        self.order = []                       # bands in the order their reduction was started (for tests)
+
+    def start(self, loss: torch.Tensor):
+        self.works, self.order = [], []
+        if not self.active:
+            return
+        for j in range(len(self.band_begin) - 1):
+            band = self.dW[self.band_begin[j]:self.band_begin[j + 1]]
+            if self.cuda:
+                self.side.wait_event(self.events[j])
+                with torch.cuda.stream(self.side):
+                    band.mul_(self.weight)
+                    self.works.append(dist.all_reduce(band, op=dist.ReduceOp.SUM, group=self.group, async_op=True))
+            else:
+                band.mul_(self.weight)
+                self.works.append(dist.all_reduce(band, op=dist.ReduceOp.SUM, group=self.group, async_op=True))
+            self.order.append(j)
+        loss.mul_(self.weight)
+        self.works.append(dist.all_reduce(loss, op=dist.ReduceOp.SUM, group=self.group, async_op=True))
+
+    def finish(self):
+        for wk in self.works:
+            wk.wait()
+        self.works = []

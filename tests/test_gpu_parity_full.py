@@ -173,6 +173,24 @@ def test_config2_whole_step_sampled_rows_and_invariants(trl, cfg2_batch, fused):
     assert row_err.max() <= 2 * TOL_GRAD, (row_err.max(), int(vsel[np.argmax(row_err)]))
 
 
+def test_config2_banded_schedule_equals_fused_step_bit_for_bit(trl, cfg2_batch):
+    """The data-parallel schedule (E kept for all rows, dW band by band over three row chunks, the
+    last one short) against the chunk-by-chunk fused step at the benchmark shape."""
+    w, batch = cfg2_batch
+    old_logp, old_lse = trl.trl_token_logprobs(batch["hidden_old"], batch["W_old"], batch["ids"], batch["lens"], w.T)
+    hrd = trl.trl_hrd_advantages(batch["r_plan"], batch["r_code"], batch["lens"], batch["bnd"], w.P, w.G, w.T)
+    args = (batch["hidden"], batch["W"], batch["ids"], batch["lens"], old_logp, old_lse, hrd["adv"], hrd["seg"], w.P, w.G, w.T)
+    ref = trl.trl_pg_step_fused(*args)
+    bands = trl.trl_dw_band_plan(w.V, w.H, 16)
+    assert len(bands) == 17
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    out = trl.trl_pg_step_fused_banded(*args, bands, rows_bound=int(batch["lens"].sum()), status=status)
+    torch.cuda.synchronize()
+    trl.check_status(status)
+    for k in ("logp", "lse", "g", "loss", "dHidden", "dW"):
+        assert torch.equal(out[k], ref[k]), k
+
+
 def test_full_size_advantages_and_loss_all_tokens(trl):
     """Steps a3 and a4 at the largest token count (config 3: 32 x 8192), every element
     against the oracle, with generator-made log-probs."""
