@@ -47,10 +47,11 @@ def test_banded_schedule_is_bit_identical_and_bands_are_final_at_their_events(tr
         e.record()
     status = torch.zeros(1, dtype=torch.int32, device=DEV)
     n_valid = int(batch["lens"].sum())
+    snap = torch.full((V, H), float("nan"), device=DEV)
+    side = torch.cuda.Stream()
+    torch.cuda.synchronize()
     out = trl.trl_pg_step_fused_banded(*args, bands, events, rows_bound=n_valid, status=status)
     # a side stream copies each band as soon as its event has fired, while later bands still run
-    side = torch.cuda.Stream()
-    snap = torch.full_like(out["dW"], float("nan"))
     for j in range(n):
         side.wait_event(events[j])
         with torch.cuda.stream(side):
