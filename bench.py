@@ -26,10 +26,11 @@ sys.path.insert(0, ROOT)
 METRIC = "scored_rollout_tokens_per_sec_fwd_bwd"
 UNIT = "tokens/s"
 WORKLOAD_ID = 2          # 8B-scale fwd+bwd: 8 prompts x 8 rollouts, T=2048, H=4096, V=151,936
-# DRAM bytes (read + write) of one tc_gemm_kernel<LSE> launch at WORKLOAD_ID, from the ncu capture of
-# the same kernel on the profile_small workload (0.897 GB: packed hidden once + W once per raster
-# band of 32 row blocks), scaled by (bands x bytes of W); the capture's summary is committed under profiles/
-LSE_TRAFFIC_BYTES = 2.85e10
+# DRAM bytes (read + write) of one tc_gemm_kernel<LSE> launch at WORKLOAD_ID, from a one-pass ncu
+# capture (dram__bytes_read.sum + dram__bytes_write.sum) of that launch inside this very command:
+# 28.14 GB read + 0.42 GB written = the packed hidden rows once + W once per raster band of 32 row
+# blocks (22 bands); the capture's summary is committed under profiles/
+LSE_TRAFFIC_BYTES = 2.856e10
 
 
 def load_peaks():

@@ -50,7 +50,9 @@ constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2;
 constexpr int RING_BYTES = 4 * (A_BYTES + B_BYTES);   // 192 KB of operand stages, cut into 3 to 6 stages
 constexpr int MAX_STAGES = 6;
 constexpr int OUT_STAGE_BYTES = 4 * 2 * 4096;   // 4 epilogue warps x 2 buffers x (32 rows x 128 B)
-constexpr int SMEM_BYTES = RING_BYTES + OUT_STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int MAX_LIST_BLOCKS = 512;               // longest list of active row blocks a CTA keeps in shared memory
+constexpr int SMEM_BYTES = RING_BYTES + OUT_STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/ +
+                           2 * MAX_LIST_BLOCKS /*active row blocks*/;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr float LOG2E = 1.4426950408889634f, LN2 = 0.6931471805599453f;
 constexpr long long WAIT_CYCLES = 4000000000LL;   // ~2-3 s at B200 clocks
@@ -494,21 +496,43 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   // ---- problem extents (identical in every thread, and in both CTAs of a pair)
   int live = p.blk_cap;
   if (p.nblk) live = max(0, min(p.nblk[0] - p.blk_off, p.blk_cap));
-  const int MB = (EPI == TC_EPI_DW) ? p.m_blocks_fixed : live;    // 128-row blocks
+  // Row blocks whose rows all have a zero gradient factor (p.blk_active) are left out.  For dW they
+  // are k-blocks, which every tile skips alike.  For dS / dHidden they are M blocks: the tiles are
+  // formed over the list of active blocks (kept in shared memory), not over all blocks with holes,
+  // so that every tile costs the same and the CTAs keep moving through K together, which is
+  // what lets them share the streamed operands in L2.
+  constexpr bool LISTED = (EPI == TC_EPI_DH || EPI == TC_EPI_DS);
+  const bool use_list = LISTED && p.blk_active != nullptr && live <= MAX_LIST_BLOCKS;
+  int n_act = live;
+  if ((EPI == TC_EPI_DW || LISTED) && p.blk_active) {
+    n_act = 0;
+    for (int i = 0; i < live; ++i) n_act += p.blk_active[i] != 0;
+  }
+  // M extent in 128-row blocks: positions in the list of active blocks when one is used
+  const int MB = (EPI == TC_EPI_DW) ? p.m_blocks_fixed : (use_list ? n_act : live);
   const int MS = (MB + MT * CG - 1) / (MT * CG);                   // tiles along M
   const int K = (EPI == TC_EPI_DW) ? live * BM : p.K;
   const int NT = (p.N + BN - 1) / BN;
   const int nkb = (K + BK - 1) / BK;
   int total = (nkb > 0) ? MS * NT : 0;
-  if (EPI == TC_EPI_DW && p.blk_active) {       // row blocks whose rows all have a zero factor add nothing to dW
-    int n_act = 0;
-    for (int i = 0; i < live; ++i) n_act += p.blk_active[i] != 0;
-    if (n_act == 0) total = 0;
-  }
+  if (n_act == 0) total = 0;
   if (total == 0 || worker >= total) return;        // the same decision in both CTAs of a pair
-  // Is M block mb worked on at all: present, and for dS / dHidden not marked inactive.
-  auto blk_on = [&](int mb) {
-    return mb < MB && (!((EPI == TC_EPI_DH || EPI == TC_EPI_DS) && p.blk_active) || p.blk_active[mb] != 0);
+  uint16_t* act_list = reinterpret_cast<uint16_t*>(gen_base + RING_BYTES + OUT_STAGE_BYTES + 256);
+  if (use_list && warp == 2) {                      // order-preserving list of the active blocks
+    int n = 0;
+    for (int i0 = 0; i0 < live; i0 += 32) {
+      const bool on = i0 + lane < live && p.blk_active[i0 + lane] != 0;
+      const unsigned m = __ballot_sync(0xffffffffu, on);
+      if (on) act_list[n + __popc(m & ((1u << lane) - 1u))] = (uint16_t)(i0 + lane);
+      n += __popc(m);
+    }
+  }
+  // M position i (accumulator j of tile ms in the CTA of rank r: i = (ms * MT + j) * CG + r) -> row block;
+  // valid after the __syncthreads below
+  auto blk_of = [&](int i) { return use_list ? (int)act_list[i] : i; };
+  // Is M position i worked on at all: present, and (without a list) not marked inactive.
+  auto pos_on = [&](int i) {
+    return i < MB && (use_list || !(LISTED && p.blk_active) || p.blk_active[i] != 0);
   };
   // Which accumulators of a tile take part (identical decision in every role and in both CTAs): an
   // accumulator spans the M blocks of all CG CTAs and runs if any of them is worked on.  Which
@@ -517,7 +541,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     int m = 0;
     for (int j = 0; j < MT; ++j)
       for (int r = 0; r < CG; ++r)
-        if (blk_on((ms * MT + j) * CG + r)) m |= 1 << j;
+        if (pos_on((ms * MT + j) * CG + r)) m |= 1 << j;
     return m;
   };
   auto kb_on = [&](int kb) { return !(EPI == TC_EPI_DW && p.blk_active) || p.blk_active[kb >> 1] != 0; };
@@ -576,7 +600,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
           for (int j = 0; j < MT; ++j) {
             if (mask & (1 << j)) {
-              const int a_row = a_row_of((ms * MT + j) * CG + rank);
+              const int pos = (ms * MT + j) * CG + rank;            // beyond the last block: any row, the result is not used
+              const int a_row = a_row_of(pos < MB ? blk_of(pos) : 0);
               if constexpr (a_is_mn(EPI)) {       // two 64(M) x 64(K) boxes
                 load(sa + j * A_BYTES, &tmA, a_row, kb * BK);
                 load(sa + j * A_BYTES + 8192, &tmA, a_row + 64, kb * BK);
@@ -666,9 +691,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       tc_fence_after();
 #pragma unroll
       for (int j = 0; j < MT; ++j) {
-        const int mb = (ms * MT + j) * CG + rank;       // this CTA's M block of accumulator j
-        if ((mask & (1 << j)) && (j % EG) == grp && blk_on(mb))
-          epilogue_tile<EPI>(p, tmem_base + (uint32_t)((acc * MT + j) * BN), quad, lane, mb, nt, wo);
+        const int pos = (ms * MT + j) * CG + rank;      // this CTA's M position of accumulator j
+        if ((mask & (1 << j)) && (j % EG) == grp && pos_on(pos))
+          epilogue_tile<EPI>(p, tmem_base + (uint32_t)((acc * MT + j) * BN), quad, lane, blk_of(pos), nt, wo);
       }
       tc_fence_before();
       if constexpr (CG == 2) mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));    // the leader's MMA issuer waits on it

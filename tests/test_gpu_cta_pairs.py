@@ -16,7 +16,7 @@ def test_parity_tests_pass_with_cta_pairs():
                            cwd=ROOT, env=env, capture_output=True, text=True)
     assert probe.returncode == 0 and "cta_group_fwd=2 cta_group_bwd=2" in probe.stdout, probe.stdout + probe.stderr
     sel = ("ragged_multi_tile or many_tiles or long_reasoning_twin or fused_step_matches_oracle or edge_cases or "
-           "smallest_legal or minimum_workspace or degenerate or all_equal or confident_policy_every")
+           "smallest_legal or minimum_workspace or degenerate or all_equal or confident_policy_every or inactive_row_blocks")
     r = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", "-m", "gpu", "tests/test_gpu_parity_small.py", "-k", sel],
                        cwd=ROOT, env=env, capture_output=True, text=True)
     assert r.returncode == 0, r.stdout[-3000:] + r.stderr[-2000:]

@@ -430,3 +430,20 @@ def test_fused_step_leaves_a_bad_id_row_out_of_loss_g_and_gradients(trl):
     assert float(out["g"][5]) == 0.0 and float(out["logp"][5]) == 0.0 and not out["dHidden"][5].any()
     assert float(out["loss"]) == float(ref["loss"]) and torch.equal(out["dHidden"], ref["dHidden"])
     assert torch.equal(out["g"], ref["g"]) and rel_fro(f64(out["dW"]), f64(ref["dW"])) < 1e-6
+
+
+@pytest.mark.parametrize("fused", [False, True])
+def test_inactive_row_blocks_between_active_ones(trl, fused):
+    """Zero-advantage groups in the middle of the batch make whole 128-row blocks inactive between
+    active ones (an odd number of them, at odd positions, plus a plan-only stretch): the gradient
+    GEMMs form their tiles over the active blocks only.  Every element against the oracle."""
+    w = synth.scaled(synth.CONFIGS[2], name="holes", P=5, G=2, T=448, H=128, V=768, len_lo=1.0, len_hi=1.0)
+    batch = synth.make_batch(w, device="cuda:0")
+    # groups 1 and 3: all-equal rewards in both classes (7 blocks of zero rows each); group 2: equal
+    # plan rewards only (its plan tokens are inactive, its code tokens are not); group 4 ends the batch inactive
+    batch["r_plan"] = torch.tensor([1.0, 0.0, 0.5, 0.5, 1.0, 1.0, 0.0, 0.0, 2.0, 2.0], device="cuda:0")
+    batch["r_code"] = torch.tensor([0.0, 1.0, 1.0, 1.0, 1.0, 0.0, 0.0, 0.0, 1.0, 1.0], device="cuda:0")
+    batch["bnd"] = torch.tensor([100, 300, 200, 10, 384, 256, 5, 440, 128, 0], dtype=torch.int32, device="cuda:0")
+    out, ref = run_and_compare(trl, w, batch=batch, fused=fused)
+    g = f64(out["g"]).reshape(w.B, w.T)
+    assert not g[2:4].any() and not g[6:10].any() and g[0].any() and g[4, 384:].any() and not g[4, :384].any()
