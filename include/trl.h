@@ -272,10 +272,13 @@ int trl_pg_loss_fwd_static(const float* logp, const float* old_logp, const float
  * counterpart in the paper. */
 unsigned long long trl_kernel_launches(void);
 
-/* Host string naming the tuning settings in effect, "cta_group_fwd=<n> cta_group_bwd=<n>": how many
- * CTAs share one tensor-core instruction in the forward and in the gradient GEMMs (1, or 2 for
- * cluster pairs).  The environment variable TRL_CTA_GROUP=1|2, read at the first call, overrides the
- * build's default for both; results are the same either way.  No counterpart in the paper. */
+/* Host string naming the tuning settings in effect,
+ * "cta_group_fwd=<n> cta_group_bwd=<n> raster_band_lse=<n> raster_band_e=<n> raster_band_dh=<n> raster_band_dw=<n>":
+ * how many CTAs share one tensor-core instruction in the forward and in the gradient GEMMs (1, or 2
+ * for cluster pairs), and how many 128-row blocks of tiles each GEMM rasterises together (the rows
+ * that stay in L2 while the other operand streams).  Environment variables, read at the first call,
+ * override the library's choices: TRL_CTA_GROUP=1|2 and TRL_RASTER_BAND_LSE / _E / _DH / _DW / _DS=<blocks>.
+ * Results are the same whatever the settings.  No counterpart in the paper. */
 const char* trl_config_string(void);
 
 /* Host string for a status code (static storage). */

@@ -150,10 +150,13 @@ size_t trl_workspace_bytes_min(int which_call, int B, int T, int H, int V, trl_d
 unsigned long long trl_kernel_launches(void) { return launches_so_far(); }
 
 const char* trl_config_string(void) {
-  static char buf[64];
+  static char buf[160];
   static std::once_flag once;
   std::call_once(once, [] {
-    snprintf(buf, sizeof(buf), "cta_group_fwd=%d cta_group_bwd=%d", tc_default_cta_group(1), tc_default_cta_group(0));
+    auto band = [](int epi, int own) { const int o = tc_raster_band_override(epi); return o ? o : own; };
+    snprintf(buf, sizeof(buf), "cta_group_fwd=%d cta_group_bwd=%d raster_band_lse=%d raster_band_e=%d raster_band_dh=%d raster_band_dw=%d",
+             tc_default_cta_group(1), tc_default_cta_group(0), band(TC_EPI_LSE, kRasterBandFwd), band(TC_EPI_E, kRasterBandFwdE),
+             band(TC_EPI_DH, kRasterBandBwd), band(TC_EPI_DW, kRasterBandBwd));
   });
   return buf;
 }

@@ -122,5 +122,6 @@ struct TcGemm {
 cudaError_t launch_tc_gemm(const TcGemm& p, cudaStream_t s);
 int tc_num_sms();
 int tc_default_cta_group(int fwd);   // CTAs per MMA in effect for the forward (1) / gradient (0) GEMMs
+int tc_raster_band_override(int epi);   // raster band in 128-row blocks from TRL_RASTER_BAND_<LSE|DS|DH|DW|E>, 0: none
 
 }  // namespace trl

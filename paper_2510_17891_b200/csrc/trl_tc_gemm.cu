@@ -34,6 +34,8 @@
 
 namespace trl {
 
+int tc_raster_band_override(int epi);
+
 namespace {
 
 // CTAs per MMA for the forward GEMMs (LSE, dS, E) and the gradient GEMMs (dHidden, dW): 1, or 2
@@ -816,7 +818,9 @@ cudaError_t launch_cg(const TcGemm& g, cudaStream_t s) {
   const int mt = (CG == 2) ? (fwd ? 1 : 2) : (g.epi == TC_EPI_LSE ? 1 : 2);     // as TileCfg
   // rows of M tiles rasterised together, so that their A rows stay in L2 while B streams: the
   // caller gives it in 128-row blocks
-  a.raster_band = (g.raster_band_blocks > 0 ? g.raster_band_blocks : 32) / (mt * CG);
+  int band_blocks = g.raster_band_blocks > 0 ? g.raster_band_blocks : 32;
+  if (const int env_band = tc_raster_band_override(g.epi)) band_blocks = env_band;
+  a.raster_band = band_blocks / (mt * CG);
   if (a.raster_band < 1) a.raster_band = 1;
   const int NT = cdiv(g.N, BN);
   const long max_tiles = (long)cdiv(g.epi == TC_EPI_DW ? g.m_blocks : g.blk_cap, mt * CG) * NT;
@@ -859,6 +863,24 @@ static int default_cta_group(bool fwd) {
 }
 
 int tc_default_cta_group(int fwd) { return default_cta_group(fwd != 0); }
+
+// Raster band (in 128-row blocks) per GEMM from the environment, for sweeps: TRL_RASTER_BAND_LSE,
+// _DS, _DH, _DW, _E (read once; 0 = the library's own choice).
+int tc_raster_band_override(int epi) {
+  static const struct Bands {
+    int v[5];
+    Bands() {
+      const char* names[5] = {"TRL_RASTER_BAND_LSE", "TRL_RASTER_BAND_DS", "TRL_RASTER_BAND_DH", "TRL_RASTER_BAND_DW",
+                              "TRL_RASTER_BAND_E"};
+      for (int i = 0; i < 5; ++i) {
+        const char* e = getenv(names[i]);
+        const int x = e ? atoi(e) : 0;
+        v[i] = (x > 0 && x <= 4096) ? x : 0;
+      }
+    }
+  } bands;
+  return (epi >= 0 && epi < 5) ? bands.v[epi] : 0;
+}
 
 cudaError_t launch_tc_gemm(const TcGemm& g, cudaStream_t s) {
   const int cg = g.cta_group > 0 ? g.cta_group : default_cta_group(!(g.epi == TC_EPI_DH || g.epi == TC_EPI_DW));

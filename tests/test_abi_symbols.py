@@ -125,3 +125,24 @@ def test_misaligned_pointers_are_rejected_on_the_host_before_any_launch():
 
     for k in (0, 1, 2, 3, 6):
         assert static(off=(k,)) == INVALID, k
+
+
+def test_config_string_names_the_tuning_settings_and_follows_the_environment(lib):
+    """Host-only: the settings string lists the library's own choices, and the environment knobs
+    (read once per process, hence child processes) replace them."""
+    import subprocess
+    import sys
+    code = "import paper_2510_17891_b200 as t; print(t.trl_config_string())"
+
+    def run(**env):
+        r = subprocess.run([sys.executable, "-c", code], cwd=ROOT, env=dict(os.environ, **env), capture_output=True, text=True)
+        assert r.returncode == 0, r.stderr
+        return dict(kv.split("=") for kv in r.stdout.split())
+
+    base = run()
+    assert base["cta_group_fwd"] == "1" and base["cta_group_bwd"] == "1"
+    assert {k: int(v) for k, v in base.items() if k.startswith("raster_band")} == {
+        "raster_band_lse": 32, "raster_band_e": 32, "raster_band_dh": 8, "raster_band_dw": 8}
+    tuned = run(TRL_CTA_GROUP="2", TRL_RASTER_BAND_LSE="48", TRL_RASTER_BAND_DW="16", TRL_RASTER_BAND_DH="nonsense")
+    assert tuned["cta_group_fwd"] == "2" and tuned["raster_band_lse"] == "48" and tuned["raster_band_dw"] == "16"
+    assert tuned["raster_band_dh"] == "8" and tuned["raster_band_e"] == "32"
