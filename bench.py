@@ -309,8 +309,9 @@ def per_ghz(tflops, sm_mhz):
 
 
 def side_run(trl, torch, synth, dev, workload_id, path, peaks, barrier, steps=3, warmup=3):
-    """A short timed run of another workload / schedule, reported under `other_runs` (not a headline)."""
-    w = synth.CONFIGS[workload_id]
+    """A short timed run of another workload / schedule, reported under `other_runs` (not a headline).
+    `workload_id` is a config number or a synth.Workload."""
+    w = synth.CONFIGS[workload_id] if isinstance(workload_id, int) else workload_id
     batch = synth.make_batch(w, device=dev)
     batch["hidden_old"] = batch["hidden"].clone()
     n_valid = int(batch["lens"].sum().item())
@@ -345,6 +346,9 @@ def main():
                     help="skip the short side runs (config 3 fused, config 2 four-call) that fill `other_runs`")
     ap.add_argument("--reductions", action="store_true",
                     help="time the two memory-bound calls (HRD advantages, surrogate loss) alone at 2^26 tokens")
+    ap.add_argument("--sweep", action="store_true",
+                    help="time the fused step on the 12 (V, H) shapes of the config-4 sweep (64 rollouts x T=1024, G=8, "
+                         "25 %% all-equal reward groups) and print one JSON line with all of them")
     ap.add_argument("--dp-allreduce", action="store_true",
                     help="data-parallel training: run the banded schedule (dW final band by band) and, with N > 1, "
                          "all-reduce every band of dW and the loss across ranks on a side stream as it becomes final")
@@ -375,6 +379,12 @@ def main():
     peaks = load_peaks()
     if args.reductions:
         run_reductions(trl, torch, dev, peaks, args)
+        return
+    if args.sweep:
+        runs = [side_run(trl, torch, synth, dev, w4, args.path, peaks, lambda: torch.cuda.synchronize(),
+                         steps=min(args.steps, 6), warmup=3)
+                for w4 in synth.sweep_workloads() if w4.G == 8]
+        print(json.dumps(dict(metric="config4_sweep_" + METRIC, unit=UNIT, path=args.path, runs=runs)))
         return
     w = synth.CONFIGS[args.workload]
     if args.small_case:
