@@ -136,6 +136,42 @@ size_t ws_bytes(int which, int B, int T, int H, int V, trl_dtype dt, bool minimu
 
 #define TRL_CUDA_OK(expr) do { if ((expr) != cudaSuccess) return TRL_ERR_CUDA; } while (0)
 
+// The gradient GEMMs are issued as several launches whose tiles fill whole waves of CTAs.  Every
+// launch starts its CTAs together again: CTAs that move through K in step find the operands their
+// neighbours stream in L2, CTAs that have drifted apart fetch them from DRAM a second time.
+constexpr int kDwBands = 16;        // launches of the dW GEMM per chunk (rounded to whole waves)
+
+// dHidden of one chunk: windows of the chunk's (active) row blocks
+cudaError_t launch_dh_in_windows(TcGemm dh, cudaStream_t s) {
+  const int win = tc_wave_aligned_blocks(dh.N);
+  if (win <= 0 || win >= dh.blk_cap) return launch_tc_gemm(dh, s);
+  for (int po = 0; po < dh.blk_cap; po += win) {
+    dh.pos_off = po; dh.pos_cap = win;
+    if (cudaError_t e = launch_tc_gemm(dh, s)) return e;
+  }
+  return cudaSuccess;
+}
+
+// dW of one chunk: bands of vocabulary rows.  `dw` describes the whole GEMM (A = E or dS [K, V],
+// m_blocks, dW, V for all V rows).
+int dw_band_plan(int V, int H, int n_bands_wanted, int32_t* band_begin);
+cudaError_t launch_dw_in_bands(TcGemm dw, int V, int H, cudaStream_t s) {
+  int32_t begin[kDwBands + 1];
+  // no band shorter than four waves of tiles: a small GEMM stays one launch
+  const long waves = (long)cdiv(V, 256) * cdiv(H, 256) / tc_num_sms();
+  const int wanted = (int)(waves / 4 < kDwBands ? waves / 4 : kDwBands);
+  const int nb = wanted >= 2 ? dw_band_plan(V, H, wanted, begin) : 1;
+  if (nb <= 1) return launch_tc_gemm(dw, s);
+  const __nv_bfloat16* A = (const __nv_bfloat16*)dw.A;
+  float* out = dw.dW;
+  for (int j = 0; j < nb; ++j) {
+    const int v0 = begin[j], vn = begin[j + 1] - v0;
+    dw.A = A + v0; dw.a_rows = vn; dw.m_blocks = cdiv(vn, kRowBlock); dw.dW = out + (size_t)v0 * H; dw.V = vn;
+    if (cudaError_t e = launch_tc_gemm(dw, s)) return e;
+  }
+  return cudaSuccess;
+}
+
 }  // namespace
 
 extern "C" {
@@ -324,7 +360,7 @@ int trl_pg_loss_bwd(const void* hidden, const void* W, const int32_t* ids, const
       dh.epi = TC_EPI_DH; dh.raster_band_blocks = kRasterBandBwd;
       dh.A = dS; dh.a_rows = R; dh.a_ld = V; dh.B = W; dh.b_rows = H; dh.b_ld = H; dh.K = V; dh.N = H;
       dh.dHidden = (__nv_bfloat16*)dHidden; dh.dh_ld = H;
-      TRL_CUDA_OK(launch_tc_gemm(dh, s));
+      TRL_CUDA_OK(launch_dh_in_windows(dh, s));
       // dW += dS^T hidden   (both operands M/N-contiguous: dS [R,V] and the chunk's packed rows [.,H])
       TcGemm dw = a;
       dw.epi = TC_EPI_DW; dw.raster_band_blocks = kRasterBandBwd;
@@ -332,7 +368,7 @@ int trl_pg_loss_bwd(const void* hidden, const void* W, const int32_t* ids, const
       dw.B = Xp + (size_t)blk_off * kRowBlock * H; dw.b_rows = H; dw.b_ld = H;
       dw.b_k = cap_rows - blk_off * kRowBlock < R ? cap_rows - blk_off * kRowBlock : R;
       dw.m_blocks = cdiv(V, kRowBlock); dw.dW = dW; dw.dw_ld = H; dw.V = V;
-      TRL_CUDA_OK(launch_tc_gemm(dw, s));
+      TRL_CUDA_OK(launch_dw_in_bands(dw, V, H, s));
     }
   } else {
     TRL_CUDA_OK(cudaMemsetAsync(dHidden, 0, N * H * 4, s));
@@ -474,13 +510,13 @@ int fused_impl(const void* hidden, const void* W, const int32_t* ids, const int3
     dh.epi = TC_EPI_DH; dh.raster_band_blocks = kRasterBandBwd;
     dh.A = E; dh.a_rows = R; dh.a_ld = V; dh.B = W; dh.b_rows = H; dh.b_ld = H; dh.K = V; dh.N = H;
     dh.dHidden = (__nv_bfloat16*)dHidden; dh.dh_ld = H; dh.row_scale = neg_alpha; dh.blk_active = blk_active;
-    TRL_CUDA_OK(launch_tc_gemm(dh, s));
+    TRL_CUDA_OK(launch_dh_in_windows(dh, s));
     // dW += E'^T (neg_alpha * hidden)
     TcGemm dw = a;
     dw.epi = TC_EPI_DW; dw.raster_band_blocks = kRasterBandBwd;
     dw.A = E; dw.a_rows = V; dw.a_ld = V; dw.B = Xs; dw.b_rows = H; dw.b_ld = H; dw.K = R; dw.N = H;
     dw.m_blocks = cdiv(V, kRowBlock); dw.dW = dW; dw.dw_ld = H; dw.V = V; dw.blk_active = blk_active;
-    TRL_CUDA_OK(launch_tc_gemm(dw, s));
+    TRL_CUDA_OK(launch_dw_in_bands(dw, V, H, s));
   }
   // loss, statistics (and g once more, identically) over all rows now that logp is complete; rows
   // whose token id is out of range stay out of it, as they stayed out of the gradients
@@ -565,7 +601,7 @@ int fused_banded(const void* hidden, const void* W, const int32_t* ids, const in
     dh.A = Ec; dh.a_rows = cb * kRowBlock; dh.a_ld = V; dh.B = W; dh.b_rows = H; dh.b_ld = H; dh.K = V; dh.N = H;
     dh.dHidden = (__nv_bfloat16*)dHidden; dh.dh_ld = H; dh.row_scale = neg_alpha + (size_t)blk_off * kRowBlock;
     dh.blk_active = blk_active + blk_off;
-    TRL_CUDA_OK(launch_tc_gemm(dh, s));
+    TRL_CUDA_OK(launch_dh_in_windows(dh, s));
   }
   for (int j = 0; j < bands.n; ++j) {
     const int v0 = bands.begin[j], vn = bands.begin[j + 1] - v0;
@@ -617,6 +653,14 @@ size_t trl_pg_step_fused_banded_workspace_bytes(int B, int T, int H, int V, int 
 }
 
 int trl_dw_band_plan(int V, int H, int n_bands_wanted, int32_t* band_begin) {
+  return dw_band_plan(V, H, n_bands_wanted, band_begin);
+}
+
+}  // extern "C"
+
+namespace {
+
+int dw_band_plan(int V, int H, int n_bands_wanted, int32_t* band_begin) {
   if (V <= 0 || H <= 0 || n_bands_wanted < 1 || !band_begin) return 0;
   // Whole 256-row tiles of dW per band, as equal as possible.  A band's launch has (tiles of the
   // band) x (tiles along H) CTA tiles; the tile count per band is rounded up to the smallest count
@@ -639,4 +683,4 @@ int trl_dw_band_plan(int V, int H, int n_bands_wanted, int32_t* band_begin) {
   return n;
 }
 
-}  // extern "C"
+}  // namespace

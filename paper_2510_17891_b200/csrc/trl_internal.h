@@ -105,6 +105,9 @@ struct TcGemm {
   int N;                                     // GEMM N extent = b_rows that are meaningful
   int m_blocks;                              // TC_EPI_DW: fixed number of 128-row blocks of A; others: from row blocks
   RowPack rb; int blk_off, blk_cap;        // chunk of row blocks
+  // all but TC_EPI_DW: this launch works on M positions [pos_off, pos_off + pos_cap) of the chunk only (pos_cap 0:
+  // all of them); a position is an entry of the list of active row blocks when blk_active is given, else a row block
+  int pos_off, pos_cap;
   int raster_band_blocks;                    // 128-row blocks rasterised together (0: default)
   int cta_group;                             // CTAs per MMA: 1, 2 (cluster pairs), 0: the build's default
   // epilogue arguments
@@ -122,6 +125,7 @@ struct TcGemm {
 cudaError_t launch_tc_gemm(const TcGemm& p, cudaStream_t s);
 int tc_num_sms();
 int tc_default_cta_group(int fwd);   // CTAs per MMA in effect for the forward (1) / gradient (0) GEMMs
+int tc_wave_aligned_blocks(int n_cols);   // M positions (128-row blocks) per launch of a gradient GEMM that fill whole waves of CTAs
 int tc_raster_band_override(int epi);   // raster band in 128-row blocks from TRL_RASTER_BAND_<LSE|DS|DH|DW|E>, 0: none
 
 }  // namespace trl

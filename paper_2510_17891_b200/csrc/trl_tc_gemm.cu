@@ -61,6 +61,7 @@ constexpr long long WAIT_CYCLES = 4000000000LL;   // ~2-3 s at B200 clocks
 
 struct TcArgs {
   int N, K, m_blocks_fixed, blk_off, blk_cap, raster_band, rows_cap, V;
+  int pos_off, pos_cap;      // window of M positions this launch works on (pos_cap 0: all)
   const int* nblk; const int* n_rows; const int* rowmap;
   const int32_t* ids; const float* lse; const float* g;
   float2* partials; float* tgt;
@@ -510,14 +511,17 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     n_act = 0;
     for (int i = 0; i < live; ++i) n_act += p.blk_active[i] != 0;
   }
-  // M extent in 128-row blocks: positions in the list of active blocks when one is used
-  const int MB = (EPI == TC_EPI_DW) ? p.m_blocks_fixed : (use_list ? n_act : live);
+  // M extent in 128-row blocks: positions in the list of active blocks when one is used.  A launch
+  // may be given a window [pos_off, pos_off + pos_cap) of those positions.
+  int MB = (EPI == TC_EPI_DW) ? p.m_blocks_fixed : (use_list ? n_act : live);
+  const int pos_off = (EPI == TC_EPI_DW || p.pos_cap <= 0) ? 0 : p.pos_off;
+  if (EPI != TC_EPI_DW && p.pos_cap > 0) MB = max(0, min(MB - pos_off, p.pos_cap));
   const int MS = (MB + MT * CG - 1) / (MT * CG);                   // tiles along M
   const int K = (EPI == TC_EPI_DW) ? live * BM : p.K;
   const int NT = (p.N + BN - 1) / BN;
   const int nkb = (K + BK - 1) / BK;
   int total = (nkb > 0) ? MS * NT : 0;
-  if (n_act == 0) total = 0;
+  if (n_act == 0 || MB == 0) total = 0;
   if (total == 0 || worker >= total) return;        // the same decision in both CTAs of a pair
   uint16_t* act_list = reinterpret_cast<uint16_t*>(gen_base + RING_BYTES + OUT_STAGE_BYTES + 256);
   if (use_list && warp == 2) {                      // order-preserving list of the active blocks
@@ -531,10 +535,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   }
   // M position i (accumulator j of tile ms in the CTA of rank r: i = (ms * MT + j) * CG + r) -> row block;
   // valid after the __syncthreads below
-  auto blk_of = [&](int i) { return use_list ? (int)act_list[i] : i; };
-  // Is M position i worked on at all: present, and (without a list) not marked inactive.
+  auto blk_of = [&](int i) { return use_list ? (int)act_list[pos_off + i] : pos_off + i; };
+  // Is M position i (of this launch's window) worked on at all: present, and (without a list) not
+  // marked inactive.
   auto pos_on = [&](int i) {
-    return i < MB && (use_list || !(LISTED && p.blk_active) || p.blk_active[i] != 0);
+    return i < MB && (use_list || !(LISTED && p.blk_active) || p.blk_active[pos_off + i] != 0);
   };
   // Which accumulators of a tile take part (identical decision in every role and in both CTAs): an
   // accumulator spans the M blocks of all CG CTAs and runs if any of them is worked on.  Which
@@ -808,7 +813,7 @@ cudaError_t launch_cg(const TcGemm& g, cudaStream_t s) {
   }
   TcArgs a;
   a.N = g.N; a.K = g.K; a.m_blocks_fixed = g.m_blocks; a.blk_off = g.blk_off; a.blk_cap = g.blk_cap;
-  a.rows_cap = g.rows_cap; a.V = g.V;
+  a.rows_cap = g.rows_cap; a.V = g.V; a.pos_off = g.pos_off; a.pos_cap = g.pos_cap;
   a.nblk = g.rb.nblk; a.n_rows = g.rb.n_rows; a.rowmap = g.rb.rowmap;
   a.ids = g.ids; a.lse = g.lse; a.g = g.g; a.partials = g.partials; a.tgt = g.tgt;
   a.dS = g.dS; a.ds_ld = g.ds_ld;
@@ -823,7 +828,8 @@ cudaError_t launch_cg(const TcGemm& g, cudaStream_t s) {
   a.raster_band = band_blocks / (mt * CG);
   if (a.raster_band < 1) a.raster_band = 1;
   const int NT = cdiv(g.N, BN);
-  const long max_tiles = (long)cdiv(g.epi == TC_EPI_DW ? g.m_blocks : g.blk_cap, mt * CG) * NT;
+  const int m_extent = g.epi == TC_EPI_DW ? g.m_blocks : (g.pos_cap > 0 && g.pos_cap < g.blk_cap ? g.pos_cap : g.blk_cap);
+  const long max_tiles = (long)cdiv(m_extent, mt * CG) * NT;
   const int slots = tc_num_sms() / CG;
   const int workers = (int)(max_tiles < (long)slots ? (max_tiles > 0 ? max_tiles : 1) : slots);
   switch (g.epi) {
@@ -863,6 +869,17 @@ static int default_cta_group(bool fwd) {
 }
 
 int tc_default_cta_group(int fwd) { return default_cta_group(fwd != 0); }
+
+// Number of 128-row M positions whose tiles (over the N extent `n_cols`) fill whole waves of the
+// persistent grid, for a gradient-type GEMM (256-row CTA tiles; 512-row pair tiles with cluster pairs).
+int tc_wave_aligned_blocks(int n_cols) {
+  const int cg = default_cta_group(false);
+  const int slots = tc_num_sms() / cg;
+  const int nt = cdiv(n_cols, BN);
+  int a = slots, b = nt;
+  while (b) { const int t = a % b; a = b; b = t; }      // a = gcd(slots, nt)
+  return (slots / a) * 2 * cg;
+}
 
 // Raster band (in 128-row blocks) per GEMM from the environment, for sweeps: TRL_RASTER_BAND_LSE,
 // _DS, _DH, _DW, _E (read once; 0 = the library's own choice).
