@@ -59,9 +59,9 @@ size_t fwd_bytes_bf16(int B, int T, int H, int V) { return row_pack_bytes(B, T) 
 size_t fwd_bytes_f32(int B, int T, int H, int V, int R) {
   return row_pack_bytes(B, T) + align_up((size_t)R * H * 4, 256) + align_up((size_t)R * V * 4, 256);
 }
-size_t bwd_fixed_bf16(int B, int T, int H, int V) {     // row packing, packed hidden, row-block activity flags
+size_t bwd_fixed_bf16(int B, int T, int H, int V) {     // row packing, packed hidden, row-block activity flags, pacing counters
   (void)V;
-  return row_pack_bytes(B, T) + xp_bytes(B, T, H) + align_up((size_t)cdiv(B * T, kRowBlock) * 4, 256);
+  return row_pack_bytes(B, T) + xp_bytes(B, T, H) + 2 * align_up((size_t)cdiv(B * T, kRowBlock) * 4, 256);
 }
 size_t bwd_per_rows_bf16(int H, int V, int R) { (void)H; return align_up((size_t)R * V * 2, 256); }   // dS chunk
 size_t bwd_bytes_f32(int B, int T, int H, int V, int R) {
@@ -141,13 +141,20 @@ size_t ws_bytes(int which, int B, int T, int H, int V, trl_dtype dt, bool minimu
 // neighbours stream in L2, CTAs that have drifted apart fetch them from DRAM a second time.
 constexpr int kDwBands = 16;        // launches of the dW GEMM per chunk (rounded to whole waves)
 
-// dHidden of one chunk: windows of the chunk's (active) row blocks
-cudaError_t launch_dh_in_windows(TcGemm dh, cudaStream_t s) {
+// k-blocks between two points at which the CTAs of the dHidden GEMM wait for one another (its
+// tiles run through K = V, thousands of k-blocks, and drift apart otherwise)
+constexpr int kPaceEvery = 64;
+
+// dHidden of one chunk: windows of the chunk's (active) row blocks.  `pace` points at zeroed
+// counters, one per launch (one per row block of the chunk is always enough).
+cudaError_t launch_dh_in_windows(TcGemm dh, unsigned* pace, cudaStream_t s) {
   const int win = tc_wave_aligned_blocks(dh.N);
+  dh.pace_ctr = pace; dh.pace_every = kPaceEvery;
   if (win <= 0 || win >= dh.blk_cap) return launch_tc_gemm(dh, s);
   for (int po = 0; po < dh.blk_cap; po += win) {
     dh.pos_off = po; dh.pos_cap = win;
     if (cudaError_t e = launch_tc_gemm(dh, s)) return e;
+    if (dh.pace_ctr) ++dh.pace_ctr;
   }
   return cudaSuccess;
 }
@@ -341,6 +348,8 @@ int trl_pg_loss_bwd(const void* hidden, const void* W, const int32_t* ids, const
     TRL_CUDA_OK(cudaMemsetAsync(dHidden, 0, N * H * 2, s));
     __nv_bfloat16* Xp = cv.take<__nv_bfloat16>((size_t)cap_rows * H);
     int* blk_active = cv.take<int>(rb.cap);
+    unsigned* pace = cv.take<unsigned>(rb.cap);
+    TRL_CUDA_OK(cudaMemsetAsync(pace, 0, (size_t)rb.cap * sizeof(unsigned), s));
     __nv_bfloat16* dS = cv.take<__nv_bfloat16>((size_t)R * V);
     launch_pack_rows_bf16((const __nv_bfloat16*)hidden, Xp, H, cap_rows, rb, 0, 0, nullptr, s);
     launch_flag_active_blocks(g, rb, blk_active, s);     // row blocks with g == 0 everywhere are skipped below
@@ -360,7 +369,7 @@ int trl_pg_loss_bwd(const void* hidden, const void* W, const int32_t* ids, const
       dh.epi = TC_EPI_DH; dh.raster_band_blocks = kRasterBandBwd;
       dh.A = dS; dh.a_rows = R; dh.a_ld = V; dh.B = W; dh.b_rows = H; dh.b_ld = H; dh.K = V; dh.N = H;
       dh.dHidden = (__nv_bfloat16*)dHidden; dh.dh_ld = H;
-      TRL_CUDA_OK(launch_dh_in_windows(dh, s));
+      TRL_CUDA_OK(launch_dh_in_windows(dh, pace + blk_off, s));
       // dW += dS^T hidden   (both operands M/N-contiguous: dS [R,V] and the chunk's packed rows [.,H])
       TcGemm dw = a;
       dw.epi = TC_EPI_DW; dw.raster_band_blocks = kRasterBandBwd;
@@ -460,6 +469,8 @@ int fused_impl(const void* hidden, const void* W, const int32_t* ids, const int3
   Carver cv(workspace);
   RowPack rb = carve_row_pack(cv.take<char>(row_pack_bytes(B, T)), B, T);
   __nv_bfloat16* Xp = cv.take<__nv_bfloat16>((size_t)cap_rows * H);
+  cv.take<int>(rb.cap);                              // (the four-call backward keeps its activity flags here)
+  unsigned* pace = cv.take<unsigned>(rb.cap);
   float* loss_partials = cv.take<float>((size_t)B * pg_loss_tiles(T) * 4);
   __nv_bfloat16* Xs = cv.take<__nv_bfloat16>((size_t)H * R);
   __nv_bfloat16* E = cv.take<__nv_bfloat16>((size_t)R * V);
@@ -471,6 +482,7 @@ int fused_impl(const void* hidden, const void* W, const int32_t* ids, const int3
   launch_build_row_pack(len, B, T, rb, status_dev, s);
   TRL_CUDA_OK(cudaMemsetAsync(dW, 0, (size_t)V * H * sizeof(float), s));
   TRL_CUDA_OK(cudaMemsetAsync(dHidden, 0, N * H * 2, s));
+  TRL_CUDA_OK(cudaMemsetAsync(pace, 0, (size_t)rb.cap * sizeof(unsigned), s));
   launch_zero_padded_f32(logp, lse, len, B, T, s);
   launch_pack_rows_bf16((const __nv_bfloat16*)hidden, Xp, H, cap_rows, rb, 0, 0, nullptr, s);
 
@@ -510,7 +522,7 @@ int fused_impl(const void* hidden, const void* W, const int32_t* ids, const int3
     dh.epi = TC_EPI_DH; dh.raster_band_blocks = kRasterBandBwd;
     dh.A = E; dh.a_rows = R; dh.a_ld = V; dh.B = W; dh.b_rows = H; dh.b_ld = H; dh.K = V; dh.N = H;
     dh.dHidden = (__nv_bfloat16*)dHidden; dh.dh_ld = H; dh.row_scale = neg_alpha; dh.blk_active = blk_active;
-    TRL_CUDA_OK(launch_dh_in_windows(dh, s));
+    TRL_CUDA_OK(launch_dh_in_windows(dh, pace + blk_off, s));
     // dW += E'^T (neg_alpha * hidden)
     TcGemm dw = a;
     dw.epi = TC_EPI_DW; dw.raster_band_blocks = kRasterBandBwd;
@@ -545,8 +557,8 @@ int fused_banded(const void* hidden, const void* W, const int32_t* ids, const in
   Carver cv(workspace);
   RowPack rb = carve_row_pack(cv.take<char>(row_pack_bytes(B, T)), B, T);
   __nv_bfloat16* Xp = cv.take<__nv_bfloat16>((size_t)cap_rows * H);
-  int* unused_flags = cv.take<int>(rb.cap);            // keeps the fixed part laid out as fused_fixed_bf16 counts it
-  (void)unused_flags;
+  cv.take<int>(rb.cap);                                // keeps the fixed part laid out as fused_fixed_bf16 counts it
+  unsigned* pace = cv.take<unsigned>(rb.cap);
   float* loss_partials = cv.take<float>((size_t)B * pg_loss_tiles(T) * 4);
   __nv_bfloat16* Xs = cv.take<__nv_bfloat16>((size_t)RB * H);
   __nv_bfloat16* E = cv.take<__nv_bfloat16>((size_t)RB * V);
@@ -557,6 +569,7 @@ int fused_banded(const void* hidden, const void* W, const int32_t* ids, const in
 
   launch_build_row_pack(len, B, T, rb, status_dev, s);
   launch_clamp_rows(rb, RB, status_dev, s);            // more valid rows than the caller's bound: flagged, the excess is dropped
+  TRL_CUDA_OK(cudaMemsetAsync(pace, 0, (size_t)rb.cap * sizeof(unsigned), s));
   TRL_CUDA_OK(cudaMemsetAsync(dW, 0, (size_t)V * H * sizeof(float), s));
   TRL_CUDA_OK(cudaMemsetAsync(dHidden, 0, N * H * 2, s));
   launch_zero_padded_f32(logp, lse, len, B, T, s);
@@ -601,7 +614,7 @@ int fused_banded(const void* hidden, const void* W, const int32_t* ids, const in
     dh.A = Ec; dh.a_rows = cb * kRowBlock; dh.a_ld = V; dh.B = W; dh.b_rows = H; dh.b_ld = H; dh.K = V; dh.N = H;
     dh.dHidden = (__nv_bfloat16*)dHidden; dh.dh_ld = H; dh.row_scale = neg_alpha + (size_t)blk_off * kRowBlock;
     dh.blk_active = blk_active + blk_off;
-    TRL_CUDA_OK(launch_dh_in_windows(dh, s));
+    TRL_CUDA_OK(launch_dh_in_windows(dh, pace + blk_off, s));
   }
   for (int j = 0; j < bands.n; ++j) {
     const int v0 = bands.begin[j], vn = bands.begin[j + 1] - v0;

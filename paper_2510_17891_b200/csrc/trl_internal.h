@@ -108,6 +108,7 @@ struct TcGemm {
   // all but TC_EPI_DW: this launch works on M positions [pos_off, pos_off + pos_cap) of the chunk only (pos_cap 0:
   // all of them); a position is an entry of the list of active row blocks when blk_active is given, else a row block
   int pos_off, pos_cap;
+  unsigned* pace_ctr; int pace_every;         // soft pacing of the CTAs every pace_every k-blocks (null: off); zero the counter before the launch
   int raster_band_blocks;                    // 128-row blocks rasterised together (0: default)
   int cta_group;                             // CTAs per MMA: 1, 2 (cluster pairs), 0: the build's default
   // epilogue arguments

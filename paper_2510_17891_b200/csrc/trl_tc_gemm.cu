@@ -62,6 +62,7 @@ constexpr long long WAIT_CYCLES = 4000000000LL;   // ~2-3 s at B200 clocks
 struct TcArgs {
   int N, K, m_blocks_fixed, blk_off, blk_cap, raster_band, rows_cap, V;
   int pos_off, pos_cap;      // window of M positions this launch works on (pos_cap 0: all)
+  unsigned* pace_ctr; int pace_every;   // soft pacing of the TMA producers (null: off); counter zeroed before the launch
   const int* nblk; const int* n_rows; const int* rowmap;
   const int32_t* ids; const float* lse; const float* g;
   float2* partials; float* tgt;
@@ -588,14 +589,36 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (lane == 0) {
       int stage = 0; uint32_t phase = 0;
       bool ok = true;
+      // Soft pacing: every pace_every k-blocks the producers of all CTAs count themselves in, and a
+      // little later each waits (bounded, falling through on expiry) until the others of its wave have
+      // reached the same point.  It keeps the CTAs within a few k-blocks of one another, so that an
+      // operand tile streamed for one of them is still in L2 when its neighbours ask for it.  No
+      // data depends on it: a producer that gives up waiting just goes on, and stops pacing.
+      bool pace = (CG == 1) && p.pace_ctr != nullptr && p.pace_every > 0 && (use_list || !(LISTED && p.blk_active));
+      const int pace_per_tile = pace ? (nkb + p.pace_every - 1) / p.pace_every : 0;
       for (int tile = worker; tile < total && ok; tile += n_workers) {
         int ms, nt;
         tile_coords(tile, MS, NT, p.raster_band, ms, nt);
         const int mask = tile_mask(ms);                        // accumulators of this tile that take part
         if (mask == 0) continue;
         const int b_row = nt * BN + rank * BN_CTA;
+        const int wave = (tile - worker) / n_workers;          // every wave before the last one is full
+        const unsigned in_wave = (unsigned)min(n_workers, total - wave * n_workers);
+        const unsigned before = (unsigned)wave * (unsigned)n_workers * (unsigned)pace_per_tile;
         for (int kb = 0; kb < nkb; ++kb) {
           if (!kb_on(kb)) continue;
+          if (pace) {
+            const int ph = kb % p.pace_every;
+            if (ph == 0) atomicAdd(p.pace_ctr, 1u);
+            if (ph == 2 || (ph < 2 && kb == nkb - 1)) {
+              const unsigned target = before + in_wave * (unsigned)(kb / p.pace_every + 1);
+              const long long t0 = clock64();
+              while (*(volatile unsigned*)p.pace_ctr < target) {
+                if (clock64() - t0 > 60000) { pace = false; break; }      // ~40 us
+                __nanosleep(200);
+              }
+            }
+          }
           if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status))) break;
           // bytes of this stage over all CTAs of the pair, expected on the leader's barrier
           if (rank == 0) mbar_expect_tx(full_bar(stage), (uint32_t)(CG * (__popc(mask) * A_BYTES + B_BYTES / CG)));
@@ -814,6 +837,7 @@ cudaError_t launch_cg(const TcGemm& g, cudaStream_t s) {
   TcArgs a;
   a.N = g.N; a.K = g.K; a.m_blocks_fixed = g.m_blocks; a.blk_off = g.blk_off; a.blk_cap = g.blk_cap;
   a.rows_cap = g.rows_cap; a.V = g.V; a.pos_off = g.pos_off; a.pos_cap = g.pos_cap;
+  a.pace_ctr = g.pace_ctr; a.pace_every = g.pace_every;
   a.nblk = g.rb.nblk; a.n_rows = g.rb.n_rows; a.rowmap = g.rb.rowmap;
   a.ids = g.ids; a.lse = g.lse; a.g = g.g; a.partials = g.partials; a.tgt = g.tgt;
   a.dS = g.dS; a.ds_ld = g.ds_ld;
