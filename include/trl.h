@@ -61,7 +61,9 @@ typedef enum {
   TRL_ERR_BAD_INDEX = 7,  /* device-detected: id, len or bnd out of range */
   TRL_ERR_TIMEOUT = 8,    /* device-detected: a bounded pipeline wait expired */
   TRL_ERR_BAD_HINT = 9,   /* device-detected: lse_hint so far off that exp(z - hint) left the fp32 range */
-  TRL_ERR_ROWS_BOUND = 10 /* device-detected: more valid rows than the caller's rows_bound (trl_pg_step_fused_banded) */
+  TRL_ERR_ROWS_BOUND = 10, /* device-detected: more valid rows than the caller's rows_bound (trl_pg_step_fused_banded) */
+  TRL_ERR_BOUNDS = 11     /* device-detected, bounds-checked debug build only: a store whose index was computed from the
+                             row packing fell outside its buffer (the store is skipped) */
 } trl_status;
 
 /* Storage type of hidden / W / dHidden.  TRL_BF16 runs on the tcgen05 tensor cores with

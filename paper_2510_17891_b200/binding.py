@@ -7,7 +7,8 @@ import torch
 TRL_F32, TRL_BF16 = 0, 1
 TRL_CALL_TOKEN_LOGPROBS, TRL_CALL_PG_LOSS_FWD, TRL_CALL_PG_LOSS_BWD, TRL_CALL_PG_STEP_FUSED = 0, 1, 2, 3
 _STATUS_BITS = {7: "index out of range (token id / len / bnd)", 8: "pipeline wait timed out",
-                9: "lse_hint out of range", 10: "more valid rows than rows_bound"}
+                9: "lse_hint out of range", 10: "more valid rows than rows_bound",
+                11: "store index outside its buffer (bounds-checked debug build)"}
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
 _lib = None
@@ -24,7 +25,9 @@ class PgConfig(ctypes.Structure):
 
 
 def lib_path():
-    return os.path.join(_PKG, "libtrl.so")
+    """libtrl.so, or with TRL_DEBUG_BUILD=1 in the environment the bounds-checked build libtrl_debug.so
+    (`python -m paper_2510_17891_b200.build --debug`)."""
+    return os.path.join(_PKG, "libtrl_debug.so" if os.environ.get("TRL_DEBUG_BUILD") == "1" else "libtrl.so")
 
 
 _vp, _sz, _i = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int

@@ -217,6 +217,7 @@ const char* trl_status_string(int status) {
     case TRL_ERR_TIMEOUT: return "pipeline wait timed out (device)";
     case TRL_ERR_BAD_HINT: return "lse_hint out of range (device)";
     case TRL_ERR_ROWS_BOUND: return "more valid rows than rows_bound (device)";
+    case TRL_ERR_BOUNDS: return "store index outside its buffer (device, debug build)";
   }
   return "unknown status";
 }
@@ -368,7 +369,7 @@ int trl_pg_loss_bwd(const void* hidden, const void* W, const int32_t* ids, const
       TcGemm dh = a;
       dh.epi = TC_EPI_DH; dh.raster_band_blocks = kRasterBandBwd;
       dh.A = dS; dh.a_rows = R; dh.a_ld = V; dh.B = W; dh.b_rows = H; dh.b_ld = H; dh.K = V; dh.N = H;
-      dh.dHidden = (__nv_bfloat16*)dHidden; dh.dh_ld = H;
+      dh.dHidden = (__nv_bfloat16*)dHidden; dh.dh_ld = H; dh.dh_rows = (long)N;
       TRL_CUDA_OK(launch_dh_in_windows(dh, pace + blk_off, s));
       // dW += dS^T hidden   (both operands M/N-contiguous: dS [R,V] and the chunk's packed rows [.,H])
       TcGemm dw = a;
@@ -521,7 +522,7 @@ int fused_impl(const void* hidden, const void* W, const int32_t* ids, const int3
     TcGemm dh = a;
     dh.epi = TC_EPI_DH; dh.raster_band_blocks = kRasterBandBwd;
     dh.A = E; dh.a_rows = R; dh.a_ld = V; dh.B = W; dh.b_rows = H; dh.b_ld = H; dh.K = V; dh.N = H;
-    dh.dHidden = (__nv_bfloat16*)dHidden; dh.dh_ld = H; dh.row_scale = neg_alpha; dh.blk_active = blk_active;
+    dh.dHidden = (__nv_bfloat16*)dHidden; dh.dh_ld = H; dh.dh_rows = (long)N; dh.row_scale = neg_alpha; dh.blk_active = blk_active;
     TRL_CUDA_OK(launch_dh_in_windows(dh, pace + blk_off, s));
     // dW += E'^T (neg_alpha * hidden)
     TcGemm dw = a;
@@ -612,7 +613,7 @@ int fused_banded(const void* hidden, const void* W, const int32_t* ids, const in
     TcGemm dh = a;
     dh.epi = TC_EPI_DH; dh.raster_band_blocks = kRasterBandBwd;
     dh.A = Ec; dh.a_rows = cb * kRowBlock; dh.a_ld = V; dh.B = W; dh.b_rows = H; dh.b_ld = H; dh.K = V; dh.N = H;
-    dh.dHidden = (__nv_bfloat16*)dHidden; dh.dh_ld = H; dh.row_scale = neg_alpha + (size_t)blk_off * kRowBlock;
+    dh.dHidden = (__nv_bfloat16*)dHidden; dh.dh_ld = H; dh.dh_rows = (long)N; dh.row_scale = neg_alpha + (size_t)blk_off * kRowBlock;
     dh.blk_active = blk_active + blk_off;
     TRL_CUDA_OK(launch_dh_in_windows(dh, pace + blk_off, s));
   }

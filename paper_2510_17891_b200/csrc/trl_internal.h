@@ -16,6 +16,23 @@ void note_launch(int n = 1);
 unsigned long long launches_so_far();
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Bounds-checked debug build (-DTRL_DEBUG_BOUNDS): stores whose index comes out of the row packing
+// (a packed row, a global row looked up in rowmap) are checked against the extent of their buffer;
+// a violation sets TRL_ERR_BOUNDS in the status word and the store is skipped.  In the normal build
+// the check is the constant true.
+#ifdef __CUDACC__
+#ifdef TRL_DEBUG_BOUNDS
+__device__ __forceinline__ bool trl_bounds_violation(int32_t* status) {
+  if (status) atomicOr(status, 1 << TRL_ERR_BOUNDS);
+  return false;
+}
+#define TRL_IN_BOUNDS(idx, extent, status) \
+  (((unsigned long long)(idx) < (unsigned long long)(extent)) ? true : trl::trl_bounds_violation(status))
+#else
+#define TRL_IN_BOUNDS(idx, extent, status) true
+#endif
+#endif
 inline int cdiv(int a, int b) { return (a + b - 1) / b; }
 
 // Row packing: the valid rows of all rollouts, in order, get consecutive packed indices
@@ -27,6 +44,7 @@ struct RowPack {
   int* row_first;  // [B+1]   packed index of each rollout's first row (exclusive prefix sum of len)
   int* rowmap;     // [cap*128] packed row -> global row b*T + t (defined for q < n_rows)
   int cap;         // ceil(B*T / 128): upper bound on nblk
+  long n_total;    // B*T: number of global rows
 };
 size_t row_pack_bytes(int B, int T);
 RowPack carve_row_pack(void* base, int B, int T);
@@ -115,7 +133,7 @@ struct TcGemm {
   const int32_t* ids; const float* lse; const float* g;
   float2* partials; float* tgt; int rows_cap;          // LSE
   __nv_bfloat16* dS; long ds_ld;                       // DS, E
-  __nv_bfloat16* dHidden; long dh_ld;                  // DH
+  __nv_bfloat16* dHidden; long dh_ld; long dh_rows;    // DH (dh_rows: rows of dHidden, for the debug build's checks)
   float* dW; long dw_ld; int V;                        // DW
   float* psum;                                         // E: row sums per vocabulary tile [n_tiles, rows_cap]
   const float* row_scale;                              // DH: optional per-scratch-row factor

@@ -24,6 +24,7 @@ RowPack carve_row_pack(void* base, int B, int T) {
   RowPack rb;
   int* p = (int*)base;
   rb.cap = cdiv(B * T, kRowBlock);
+  rb.n_total = (long)B * T;
   rb.nblk = p;
   rb.n_rows = p + 1;
   rb.row_first = p + 2;
@@ -69,18 +70,22 @@ __global__ void build_row_pack_kernel(const int32_t* __restrict__ len, int B, in
   }
 }
 
-__global__ void __launch_bounds__(256) fill_rowmap_kernel(const int32_t* __restrict__ len, int B, int T, RowPack rb) {
+__global__ void __launch_bounds__(256) fill_rowmap_kernel(const int32_t* __restrict__ len, int B, int T, RowPack rb,
+                                                          int32_t* status) {
   const size_t n = (size_t)blockIdx.x * 256 + threadIdx.x;
   if (n >= (size_t)B * T) return;
   const int b = (int)(n / T), t = (int)(n % T);
-  if (t < max(0, min(len[b], T))) rb.rowmap[rb.row_first[b] + t] = (int)n;
+  if (t < max(0, min(len[b], T))) {
+    const long q = (long)rb.row_first[b] + t;
+    if (TRL_IN_BOUNDS(q, (long)rb.cap * kRowBlock, status)) rb.rowmap[q] = (int)n;
+  }
 }
 
 void launch_build_row_pack(const int32_t* len, int B, int T, RowPack rb, int32_t* status, cudaStream_t s) {
   build_row_pack_kernel<<<1, 1024, 0, s>>>(len, B, T, rb, status);
   note_launch();
   const size_t N = (size_t)B * T;
-  fill_rowmap_kernel<<<(unsigned)((N + 255) / 256), 256, 0, s>>>(len, B, T, rb);
+  fill_rowmap_kernel<<<(unsigned)((N + 255) / 256), 256, 0, s>>>(len, B, T, rb, status);
   note_launch();
 }
 
@@ -483,13 +488,13 @@ __global__ void __launch_bounds__(128) fused_merge_kernel(FusedMergeArgs a) {
     if (!(sum > 0.f) || !isfinite(sum)) flag_status(a.status, TRL_ERR_BAD_HINT);
     const float lse = c + logf(sum);
     const float lp = id_ok ? zt - lse : 0.f;
-    a.logp[n] = lp;
-    a.lse[n] = lse;
+    const bool n_ok = TRL_IN_BOUNDS(n, a.rb.n_total, a.status);
+    if (n_ok) { a.logp[n] = lp; a.lse[n] = lse; }
     const int L = max(0, min(a.len[b], a.T));
     const float inv = a.cfg.agg_mode == 1 ? 1.0f / (float)a.rb.n_rows[0] : 1.0f / ((float)a.P * (float)a.G * (float)L);
     const TokenTerm tt = surrogate_token(lp, a.old_logp[n], a.adv[n], a.seg[n], a.cfg, inv);
     gn = id_ok ? tt.g : 0.f;
-    a.g[n] = gn;
+    if (n_ok) a.g[n] = gn;
     if (gn != 0.f) a.E[(size_t)r * a.V + id] = __float2bfloat16_rn(-s_excl);
     gn = -gn * expf(c - lse);
   }
@@ -564,7 +569,7 @@ __global__ void __launch_bounds__(256) row_lse_f32_kernel(const float* __restric
   float l = 0.f;
   for (int v = threadIdx.x; v < V; v += 256) l += expf(row[v] - m);
   l = block_reduce(l, false, sh);
-  if (threadIdx.x == 0) {
+  if (threadIdx.x == 0 && TRL_IN_BOUNDS(n, rb.n_total, status)) {
     const float L = m + logf(l);
     lse[n] = L;
     const int id = ids[n];
@@ -603,7 +608,7 @@ __global__ void scatter_rows_f32_kernel(const float* __restrict__ dHp, float* __
                                         RowPack rb, int blk_off) {
   const int r = blockIdx.x;
   const long n = scratch_row_to_global(rb, blk_off, r);
-  if (n < 0) return;
+  if (n < 0 || !TRL_IN_BOUNDS(n, rb.n_total, (int32_t*)nullptr)) return;
   for (int h = threadIdx.x; h < H; h += blockDim.x) dHidden[(size_t)n * H + h] = dHp[(size_t)r * H + h];
 }
 void launch_scatter_rows_f32(const float* dHp, float* dHidden, int H, int R, RowPack rb, int blk_off,

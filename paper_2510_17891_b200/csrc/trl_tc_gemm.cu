@@ -67,7 +67,7 @@ struct TcArgs {
   const int32_t* ids; const float* lse; const float* g;
   float2* partials; float* tgt;
   __nv_bfloat16* dS; long ds_ld;
-  __nv_bfloat16* dHidden; long dh_ld;
+  __nv_bfloat16* dHidden; long dh_ld; long dh_rows;
   float* dW; long dw_ld;
   float* psum; const float* row_scale;
   const int* blk_active;     // per row block of the chunk: 0 = every row has a zero gradient factor (may be null)
@@ -336,8 +336,10 @@ __device__ __forceinline__ void epilogue_tile(const TcArgs& p, uint32_t tmem_acc
       }
     }
     const size_t prow = (size_t)prow_i;
-    p.partials[(size_t)nt * p.rows_cap + prow] = make_float2(m2 * LN2, l);
-    if (has) p.tgt[prow] = tg;
+    if (TRL_IN_BOUNDS(prow, p.rows_cap, p.status)) {
+      p.partials[(size_t)nt * p.rows_cap + prow] = make_float2(m2 * LN2, l);
+      if (has) p.tgt[prow] = tg;
+    }
   } else if constexpr (EPI == TC_EPI_DS) {
     const int prow_i = (p.blk_off + mb) * BM + r;          // packed row
     const bool valid = prow_i < p.n_rows[0];
@@ -409,20 +411,23 @@ __device__ __forceinline__ void epilogue_tile(const TcArgs& p, uint32_t tmem_acc
       }
       wo.put<false>(w, n0 + c0, mb * BM + quad * 32);
     }
-    p.psum[(size_t)nt * p.rows_cap + srow] = sum;
-    if (has) p.tgt[srow] = tg;
+    if (TRL_IN_BOUNDS(srow, p.rows_cap, p.status)) {
+      p.psum[(size_t)nt * p.rows_cap + srow] = sum;
+      if (has) p.tgt[srow] = tg;
+    }
   } else if constexpr (EPI == TC_EPI_DH) {
     const int prow_i = (p.blk_off + mb) * BM + r;          // packed row
     const bool valid = prow_i < p.n_rows[0];
     const long grow = valid ? (long)p.rowmap[prow_i] : 0;
     const float rs = p.row_scale ? p.row_scale[(size_t)mb * BM + r] : 1.0f;
+    const bool row_ok = TRL_IN_BOUNDS(grow, p.dh_rows, p.status);     // constant true outside the debug build
     __nv_bfloat16* out = p.dHidden + (size_t)grow * p.dh_ld;
     for (int c0 = 0; c0 < BN; c0 += 32) {
       const int ncl = p.N - (n0 + c0);
       if (ncl <= 0) break;
       tc_ld32(taddr + c0, v);
       tc_wait_ld();
-      if (valid) {
+      if (valid && row_ok) {
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
           if (q * 8 < ncl) {
@@ -841,7 +846,7 @@ cudaError_t launch_cg(const TcGemm& g, cudaStream_t s) {
   a.nblk = g.rb.nblk; a.n_rows = g.rb.n_rows; a.rowmap = g.rb.rowmap;
   a.ids = g.ids; a.lse = g.lse; a.g = g.g; a.partials = g.partials; a.tgt = g.tgt;
   a.dS = g.dS; a.ds_ld = g.ds_ld;
-  a.dHidden = g.dHidden; a.dh_ld = g.dh_ld; a.dW = g.dW; a.dw_ld = g.dw_ld; a.status = g.status;
+  a.dHidden = g.dHidden; a.dh_ld = g.dh_ld; a.dh_rows = g.dh_rows; a.dW = g.dW; a.dw_ld = g.dw_ld; a.status = g.status;
   a.psum = g.psum; a.row_scale = g.row_scale; a.blk_active = g.blk_active;
   const bool fwd = (g.epi == TC_EPI_LSE || g.epi == TC_EPI_E || g.epi == TC_EPI_DS);
   const int mt = (CG == 2) ? (fwd ? 1 : 2) : (g.epi == TC_EPI_LSE ? 1 : 2);     // as TileCfg

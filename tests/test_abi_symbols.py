@@ -146,3 +146,12 @@ def test_config_string_names_the_tuning_settings_and_follows_the_environment(lib
     tuned = run(TRL_CTA_GROUP="2", TRL_RASTER_BAND_LSE="48", TRL_RASTER_BAND_DW="16", TRL_RASTER_BAND_DH="nonsense")
     assert tuned["cta_group_fwd"] == "2" and tuned["raster_band_lse"] == "48" and tuned["raster_band_dw"] == "16"
     assert tuned["raster_band_dh"] == "8" and tuned["raster_band_e"] == "32"
+
+
+def test_bounds_checked_build_compiles_and_exports_the_same_symbols():
+    from paper_2510_17891_b200 import build
+    dbg = ctypes.CDLL(build.build(debug=True))
+    for n in _declared():
+        assert hasattr(dbg, n), n
+    dbg.trl_status_string.restype = ctypes.c_char_p
+    assert b"debug build" in dbg.trl_status_string(11)
